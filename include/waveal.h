@@ -1,0 +1,178 @@
+/* waveal - WaveAlign-scheduled block-sparse attention for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library.  Two groups of calls:
+ *   planning   waveal_plan_bitmap / waveal_plan_csr : block mask -> per-head execution order
+ *              of the query blocks (Algorithm 2 of the WaveAlign paper, with the adaptive
+ *              skip of Section 4.5 in front);
+ *   attention  waveal_bsattn_fwd : block-sparse FlashAttention-style forward (Sections
+ *              2.2-2.3) whose persistent CTAs walk that order head by head.
+ *
+ * Conventions for every call
+ *   - "dev" pointers are device pointers on the current CUDA device, "host" pointers are
+ *     host pointers.  The caller owns every buffer and the stream.
+ *   - The library allocates no device memory, never frees and never synchronises (unless a
+ *     call's comment says otherwise); all work is enqueued on `cuda_stream` (a cudaStream_t
+ *     passed as void*, NULL = the default stream).
+ *   - A problem the host can detect returns a non-zero status BEFORE anything is enqueued
+ *     and leaves the outputs untouched; waveal_last_error() then describes it.
+ *   - Problems only the device can detect (a bounded wait that ran out, an index out of
+ *     range) are written to the `dev_status` words; the kernel leaves cleanly, nothing traps.
+ *   - heads = batch * heads flattened; every head has its own mask (Algorithm 2 input
+ *     M in {0,1}^{H x M_B x N_B}).
+ *   - Mask bitmap: row-major uint64 [heads][n_q_blocks][ceil(n_kv_blocks/64)]; bit (j & 63)
+ *     of word (j >> 6) of row i is M[i][j]; padding bits must be zero.
+ *   - Index lists (CSR over the flattened (head, query block) axis): kv_row_ptr int32
+ *     [heads*n_q_blocks + 1], kv_block_indices int32 [nnz], ascending and unique inside a row.
+ *   - Execution order: row_order int32 [heads][n_q_blocks]; row_order[h][p] is the query
+ *     block executed at position p of head h (the index-list form of P_h in Algorithm 2).
+ */
+#ifndef WAVEAL_H_
+#define WAVEAL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  WAVEAL_OK = 0,
+  WAVEAL_ERR_INVALID_ARG = 1,   /* NULL pointer, non-positive size, misaligned pointer/stride */
+  WAVEAL_ERR_UNSUPPORTED = 2,   /* head_dim / block size / dtype / device not supported      */
+  WAVEAL_ERR_WORKSPACE = 3,     /* workspace missing or too small                             */
+  WAVEAL_ERR_BAD_MASK = 4,      /* device-side: index out of range / unsorted                 */
+  WAVEAL_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed                          */
+  WAVEAL_ERR_TIMEOUT = 6        /* device-side: a bounded wait ran out                        */
+} waveal_status;
+
+/* Which stages run (Section 6.5 ablation: Original, O+S1, O+S2, O+S1+S2). */
+typedef enum {
+  WAVEAL_AUTO = 0,           /* guard decides per head; a skipped head keeps natural order */
+  WAVEAL_FORCE_REORDER = 1,  /* Stage 1 + Stage 2 on every head                            */
+  WAVEAL_FORCE_NATURAL = 2,  /* identity order on every head                               */
+  WAVEAL_STAGE1_ONLY = 3,    /* angular order only                                         */
+  WAVEAL_STAGE2_ONLY = 4     /* natural order cut into waves, each sorted by block count   */
+} waveal_mode;
+
+/* skip_flags bits */
+#define WAVEAL_FLAG_SKIPPED 1u        /* this head's row_order is the identity (skip applied) */
+#define WAVEAL_FLAG_SHORT_SEQ 2u      /* one head's K+V fit the L2 budget (Section 4.5, case 1) */
+#define WAVEAL_FLAG_TOO_SPARSE 4u     /* too little work to amortise reordering (case 2)        */
+#define WAVEAL_FLAG_ALREADY_LOCAL 8u  /* natural-order waves already overlap (case 3)           */
+
+typedef struct waveal_plan_desc {
+  int32_t heads;          /* batch*heads                                                      */
+  int32_t n_q_blocks;     /* M_B (Section 4.2)                                                */
+  int32_t n_kv_blocks;    /* N_B                                                              */
+  int32_t wave_size;      /* W = SMs x resident CTAs (Section 6.1); 0 = this device's SM count */
+  int32_t svd_iters;      /* T of Algorithm 1 (paper: 5-15)                                   */
+  int32_t mode;           /* waveal_mode                                                      */
+  uint64_t seed;          /* seed of the start block of Algorithm 1                           */
+  /* guard thresholds, all integer comparisons (the "offline profile" of Section 4.5):       */
+  int64_t kv_bytes_per_head; /* bytes of K plus V of one head; 0 disables the short-seq test */
+  int64_t l2_bytes;          /* cache size the test compares with; 0 = query the device      */
+  int32_t l2_fit_num, l2_fit_den;  /* short-seq: kv_bytes*den <= l2_bytes*num                */
+  int32_t min_density_ppm;         /* too-sparse: nnz*1e6 < ppm*M_B*N_B ...                  */
+  int32_t local_num, local_den;    /* already-local: 2*ov_nat*den >= num*pair2               */
+  int64_t min_nnz;                 /* ... or nnz < min_nnz (per head)                        */
+} waveal_plan_desc;
+
+/* Optional and required outputs of a plan call (all dev pointers; NULL = not wanted,
+ * except row_order). */
+typedef struct waveal_plan_out {
+  int32_t* row_order;   /* [heads][M_B]  required                                            */
+  int32_t* row_nnz;     /* [heads][M_B]  n_i = sum_j M_ij (Section 2.2)                      */
+  uint8_t* skip_flags;  /* [heads]       WAVEAL_FLAG_* bits                                  */
+  int32_t* col_count;   /* [heads][N_B]  c = M^T 1 (Algorithm 1)                             */
+  int32_t* order1;      /* [heads][M_B]  Stage-1 order before the per-wave sort              */
+  double* embedding;    /* [heads][M_B][2]  u_1, u_2 of Algorithm 1 (zeros for skipped heads) */
+  int64_t* stats;       /* [heads][4]    nnz, ov_nat, pair2, 0 (guard statistics)            */
+  int32_t* dev_status;  /* [4] {code, site, head, aux}; written only on a device-side failure
+                           (an index list entry out of range); the caller zeroes it          */
+} waveal_plan_out;
+
+/* Fills `desc` with the library defaults (T = 10, AUTO, default guard thresholds);
+ * heads / block counts stay 0 for the caller to set.  Host-only, no CUDA call. */
+void waveal_plan_desc_default(waveal_plan_desc* desc /*host*/);
+
+/* Bytes of device workspace a plan call needs (the same for the bitmap and CSR entry).
+ * Host-only. */
+waveal_status waveal_plan_workspace_bytes(const waveal_plan_desc* desc /*host*/, size_t* bytes /*host*/);
+
+/* Algorithm 2 from a bitmap mask.  Steps, all on the device: row block counts and column
+ * counts (Algorithm 1 step 1, Algorithm 2 Stage 2), guard statistics and decision
+ * (Section 4.5), T centred subspace iterations + Rayleigh-Ritz ordering (Algorithm 1),
+ * polar angle (Eq. 4), angular sort, wave-sized buckets, descending-count sort per bucket.
+ * ws: dev workspace of at least waveal_plan_workspace_bytes bytes, 256-byte aligned.
+ * No host synchronisation: the skip decision is consumed on the device. */
+waveal_status waveal_plan_bitmap(const waveal_plan_desc* desc /*host*/, const uint64_t* mask_bits /*dev*/,
+                                 void* ws /*dev*/, size_t ws_bytes, const waveal_plan_out* out /*host struct of dev ptrs*/,
+                                 void* cuda_stream);
+
+/* Same from index lists; the bitmap is built in the workspace first. */
+waveal_status waveal_plan_csr(const waveal_plan_desc* desc /*host*/, const int32_t* kv_row_ptr /*dev*/,
+                              const int32_t* kv_block_indices /*dev*/, void* ws /*dev*/, size_t ws_bytes,
+                              const waveal_plan_out* out, void* cuda_stream);
+
+/* Bitmap -> index lists, so that the attention kernel has one input format.
+ * kv_row_ptr_out: dev int32 [heads*n_q_blocks + 1] (always written).
+ * kv_block_indices_out: dev int32 [capacity] or NULL to compute only the row pointers;
+ * entries beyond `capacity` are not written (the caller sizes it from kv_row_ptr_out's last
+ * entry or from an upper bound).  ws: dev scratch of at least
+ * (heads*n_q_blocks + 1) * 4 bytes. */
+waveal_status waveal_bitmap_to_csr(int32_t heads, int32_t n_q_blocks, int32_t n_kv_blocks,
+                                   const uint64_t* mask_bits /*dev*/, int32_t* kv_row_ptr_out /*dev*/,
+                                   int32_t* kv_block_indices_out /*dev or NULL*/, int64_t capacity,
+                                   void* ws /*dev*/, size_t ws_bytes, void* cuda_stream);
+
+typedef struct waveal_attn_desc {
+  int32_t heads;            /* batch*heads; K/V heads == Q heads                              */
+  int32_t seq_q, seq_kv;    /* true (unpadded) lengths                                        */
+  int32_t head_dim;         /* 64 or 128                                                      */
+  int32_t block_q, block_kv;/* 64 or 128, equal; the mask's block size (Section 2.2)          */
+  int64_t q_stride[2], k_stride[2], v_stride[2], o_stride[2]; /* elements: {head, token}; head_dim contiguous */
+  int32_t order_heads_interleaved; /* 0 = heads run one after another (Section 5, sequential
+                                      heads); 1 = position-major across heads (parallel heads) */
+  int32_t reserved;
+} waveal_attn_desc;
+
+/* Bytes of device workspace waveal_bsattn_fwd needs (ticket counter + abort flag).  Host-only. */
+waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* desc /*host*/, size_t* bytes /*host*/);
+
+/* Block-sparse attention forward, bf16 in / fp32 accumulate / bf16 out (Sections 2.1-2.3):
+ * for query block i of head h, O = softmax(scale * Q_i K_sel^T) V_sel over the tokens of
+ * the K/V blocks listed for (h, i), visited in the listed (ascending) order.
+ * Persistent CTAs take (head, position) tickets in head-major order and process query
+ * block row_order[h][position] (Algorithm 2 output; NULL = natural order); each output
+ * tile is written at its original rows, so no inverse permutation pass exists.
+ * Q, K, V, O: dev bf16, 16-byte aligned, strides multiples of 8 elements, head_dim
+ * contiguous; query tokens >= seq_q are not written; keys >= seq_kv are ignored.
+ * lse: dev float [heads][seq_q] or NULL (natural-log sum-exp per query token; -inf for a
+ * query block with an empty list, whose O is 0).
+ * scale <= 0 means 1/sqrt(head_dim).
+ * ws: dev workspace (waveal_bsattn_workspace_bytes), 16-byte aligned.
+ * dev_status: dev int32 [4] or NULL: {code, site, block, aux}; written only on a device-side
+ * failure (the caller zeroes it).
+ * The first call in a process also looks up a driver entry point (no allocation). */
+waveal_status waveal_bsattn_fwd(const waveal_attn_desc* desc /*host*/, const void* Q, const void* K, const void* V,
+                                void* O, float* lse, const int32_t* kv_row_ptr /*dev*/,
+                                const int32_t* kv_block_indices /*dev*/, const int32_t* row_order /*dev or NULL*/,
+                                float scale, void* ws /*dev*/, size_t ws_bytes, int32_t* dev_status /*dev or NULL*/,
+                                void* cuda_stream);
+
+/* Number of query-block tasks the attention kernel keeps in flight on the current device
+ * (SM count x CTAs per SM): the W to plan with (Section 6.1).  Returns <= 0 on failure. */
+int32_t waveal_default_wave_size(void);
+
+/* Number of kernel launches the last successful call on this thread enqueued. */
+int32_t waveal_last_launch_count(void);
+
+const char* waveal_status_string(waveal_status s);
+/* Thread-local description of the last failure on this thread ("" if none). */
+const char* waveal_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WAVEAL_H_ */

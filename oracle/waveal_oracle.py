@@ -251,14 +251,16 @@ DEFAULT_GUARD = dict(kv_bytes_per_head=0, l2_bytes=0, l2_fit_num=1, l2_fit_den=2
 
 def guard_flags(mask: np.ndarray, wave: int, g: Dict[str, int]) -> int:
     """Adaptive skip (Section 4.5), decided before reordering, as integer comparisons:
-    short sequence: kv_bytes * den <= l2_bytes * num (one head's K+V fit the cache budget);
+    short sequence: kv_bytes * den <= l2_bytes * num (one head's K+V fit the cache budget;
+    tested only when both byte counts are positive);
     too sparse: nnz < min_nnz or nnz * 1e6 < min_density_ppm * M_B * N_B;
     already local: 2 * ov_nat * local_den >= local_num * pair2 (and pair2 > 0).
     Returns the reason bits (FLAG_SHORT_SEQ | FLAG_TOO_SPARSE | FLAG_ALREADY_LOCAL)."""
     st = guard_stats(mask, wave)
     m_b, n_b = mask.shape
     flags = 0
-    if g["l2_bytes"] > 0 and g["kv_bytes_per_head"] * g["l2_fit_den"] <= g["l2_bytes"] * g["l2_fit_num"]:
+    if g["kv_bytes_per_head"] > 0 and g["l2_bytes"] > 0 and \
+            g["kv_bytes_per_head"] * g["l2_fit_den"] <= g["l2_bytes"] * g["l2_fit_num"]:
         flags |= FLAG_SHORT_SEQ
     if st["nnz"] < g["min_nnz"] or st["nnz"] * 1_000_000 < g["min_density_ppm"] * m_b * n_b:
         flags |= FLAG_TOO_SPARSE

@@ -1,0 +1,61 @@
+"""Helpers for the GPU parity tests: move a synthetic workload to the device and sample
+tasks for the oracle."""
+from __future__ import annotations
+
+import math
+from typing import List, Sequence
+
+import numpy as np
+import torch
+
+from paper_2609_34814_b200 import binding as wb
+from paper_2609_34814_b200 import inputs as I
+
+
+class Workload:
+    """Masks, index lists and Q/K/V of one config on the device (heads subset optional)."""
+
+    def __init__(self, cfg: I.Config, heads: Sequence[int] = None, device="cuda", need_tensors=True):
+        self.cfg = cfg
+        self.heads = list(range(cfg.heads)) if heads is None else list(heads)
+        self.masks = [I.make_mask(cfg, h) for h in self.heads]
+        self.bitmap_np = np.stack([I.mask_to_bitmap(m) for m in self.masks])
+        self.ptr_np, self.idx_np = I.masks_to_csr(self.masks)
+        self.bitmap = torch.from_numpy(self.bitmap_np.view(np.int64)).to(device)
+        self.ptr = torch.from_numpy(self.ptr_np).to(device)
+        self.idx = torch.from_numpy(self.idx_np).to(device)
+        self.nnz = int(self.ptr_np[-1])
+        if need_tensors:
+            H = len(self.heads)
+            self.q, self.k, self.v = (torch.empty((H, cfg.seq_pad, cfg.head_dim), dtype=torch.bfloat16, device=device)
+                                      for _ in range(3))
+            for i, h in enumerate(self.heads):
+                for name, dst in (("q", self.q), ("k", self.k), ("v", self.v)):
+                    dst[i].copy_(I.make_head_tensor(cfg, name, h))
+            self.o = torch.zeros_like(self.q)
+
+    def head_f64(self, which: str, local_head: int) -> np.ndarray:
+        return I.bf16_to_f64(I.make_head_tensor(self.cfg, which, self.heads[local_head]))
+
+    def attn_desc(self, interleaved=False):
+        c = self.cfg
+        return wb.attn_desc(self.q, self.k, self.v, self.o, c.seq, c.seq, c.block, interleaved)
+
+    def flops(self) -> float:
+        c = self.cfg
+        return 4.0 * c.block * c.block * c.head_dim * self.nnz
+
+
+def run_attention(w: Workload, row_order=None, lse=None, out=None, scale=0.0, interleaved=False):
+    """One waveal_bsattn_fwd call; returns (O, dev_status list)."""
+    o = w.o if out is None else out
+    st = torch.zeros(4, dtype=torch.int32, device=o.device)
+    d = wb.attn_desc(w.q, w.k, w.v, o, w.cfg.seq, w.cfg.seq, w.cfg.block, interleaved)
+    wb.bsattn_fwd(d, w.q, w.k, w.v, o, w.ptr, w.idx, row_order=row_order, lse=lse, scale=scale, dev_status=st)
+    torch.cuda.synchronize()
+    return o, st.tolist()
+
+
+def error_stats(gpu: np.ndarray, ref: np.ndarray):
+    d = np.abs(gpu.astype(np.float64) - ref)
+    return float(d.max()), float(d.mean())
