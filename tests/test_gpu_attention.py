@@ -1,0 +1,178 @@
+"""GPU parity of the block-sparse attention kernel against the CPU oracle (through the C ABI).
+
+Tolerance (bf16 inputs, fp32 accumulation, bf16 output): max-abs 1e-2, mean-abs 1e-3."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import waveal_oracle as wo
+from paper_2609_34814_b200 import binding as wb
+from paper_2609_34814_b200 import inputs as I
+from gpu_util import Workload, run_attention, error_stats
+
+pytestmark = pytest.mark.gpu
+MAX_ABS, MEAN_ABS = 1e-2, 1e-3
+
+
+def _oracle_head(w, li, scale=None):
+    cfg = w.cfg
+    Q, K, V = (w.head_f64(x, li) for x in "qkv")
+    return wo.block_sparse_attention(Q, K, V, w.masks[li], cfg.block, cfg.block, cfg.seq, cfg.seq, scale)
+
+
+def _small(name, frames, heads, **kw):
+    cfg = I.CONFIGS[name]
+    return dataclasses.replace(cfg, frames=frames, seq=frames * cfg.frame_tokens - kw.pop("cut", 0), heads=heads,
+                               name=f"{name}_small", **kw)
+
+
+SMALL = [
+    ("tiny", I.CONFIGS["tiny"]),                              # 64x64 blocks, D=64, every row
+    ("wan480p_r", _small("wan480p", 3, 2)),                   # 128x128, D=128, 4680 tokens: ragged last block (72)
+    ("wan720p_r", _small("wan720p", 2, 2, cut=37)),           # 7163 tokens: ragged (123)
+    ("ltx_r", _small("ltxmixed", 3, 2, cut=10)),              # 64x64 blocks, D=128, ragged, sink rows
+    ("b128_d64", dataclasses.replace(_small("wan480p", 2, 2), head_dim=64)),
+]
+
+
+@pytest.mark.parametrize("name,cfg", SMALL, ids=[s[0] for s in SMALL])
+def test_attention_full_parity_small(name, cfg):
+    w = Workload(cfg)
+    lse = torch.full((cfg.heads, cfg.seq), float("nan"), dtype=torch.float32, device="cuda")
+    w.o.fill_(float("nan"))
+    o, st = run_attention(w, lse=lse)
+    assert st == [0, 0, 0, 0]
+    for li in range(cfg.heads):
+        ref, ref_lse = _oracle_head(w, li)
+        g = o[li, :cfg.seq].float().cpu().numpy()
+        mx, mean = error_stats(g, ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS, (name, li, mx, mean)
+        assert np.abs(lse[li].cpu().numpy() - ref_lse).max() < 2e-3
+        # padded query rows (beyond seq) are never written
+        if cfg.seq_pad > cfg.seq:
+            assert torch.isnan(o[li, cfg.seq:].float()).all()
+
+
+def test_output_is_bitwise_invariant_under_row_order():
+    # Section 4.1: reordering changes only the execution order; Table 3: outputs identical
+    cfg = _small("wan720p", 4, 3)
+    w = Workload(cfg)
+    base, st = run_attention(w, out=torch.zeros_like(w.o))
+    assert st[0] == 0
+    d = wb.plan_desc_default(heads=3, n_q_blocks=cfg.n_blocks, n_kv_blocks=cfg.n_blocks, wave_size=16,
+                             mode=wb.FORCE_REORDER, seed=5)
+    plan = wb.plan_bitmap(d, w.bitmap)
+    out1, st = run_attention(w, row_order=plan.row_order, out=torch.zeros_like(w.o))
+    assert st[0] == 0 and torch.equal(base, out1)
+    rng = np.random.default_rng(0)
+    perm = np.stack([rng.permutation(cfg.n_blocks) for _ in range(3)]).astype(np.int32)
+    out2, st = run_attention(w, row_order=torch.from_numpy(perm).cuda(), out=torch.zeros_like(w.o))
+    assert st[0] == 0 and torch.equal(base, out2)
+    out3, st = run_attention(w, row_order=plan.row_order, out=torch.zeros_like(w.o), interleaved=True)
+    assert st[0] == 0 and torch.equal(base, out3)
+    # run-to-run determinism
+    out4, _ = run_attention(w, out=torch.zeros_like(w.o))
+    assert torch.equal(base, out4)
+
+
+def test_empty_rows_scale_and_strides():
+    cfg = _small("wan480p", 2, 2)
+    w = Workload(cfg)
+    # empty list for some rows: O = 0, LSE = -inf
+    masks = [m.copy() for m in w.masks]
+    masks[0][3, :] = False
+    masks[1][0, :] = False
+    w.masks = masks
+    ptr, idx = I.masks_to_csr(masks)
+    w.ptr, w.idx = torch.from_numpy(ptr).cuda(), torch.from_numpy(idx).cuda()
+    # strided layout: heads interleaved in one [tokens, heads, D] buffer
+    buf = torch.empty((cfg.seq_pad, 2, 3, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
+    for t, src in enumerate((w.q, w.k, w.v)):
+        buf[:, :, t].copy_(src.permute(1, 0, 2))
+    w.q, w.k, w.v = (buf[:, :, t].permute(1, 0, 2) for t in range(3))
+    o = torch.full((2, cfg.seq_pad, cfg.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((2, cfg.seq), dtype=torch.float32, device="cuda")
+    scale = 0.05
+    o, st = run_attention(w, out=o, lse=lse, scale=scale)
+    assert st[0] == 0
+    b = cfg.block
+    assert (o[0, 3 * b:4 * b] == 0).all() and torch.isinf(lse[0, 3 * b:4 * b]).all()
+    assert (o[1, :b] == 0).all() and (lse[1, :b] < 0).all()
+    for li in range(2):
+        ref, ref_lse = _oracle_head(w, li, scale)
+        mx, mean = error_stats(o[li, :cfg.seq].float().cpu().numpy(), ref)
+        assert mx <= MAX_ABS and mean <= MEAN_ABS
+        fin = np.isfinite(ref_lse)
+        assert np.abs(lse[li].cpu().numpy()[fin] - ref_lse[fin]).max() < 2e-3
+
+
+def test_closed_forms_on_gpu():
+    cfg = _small("wan480p", 2, 1)
+    w = Workload(cfg)
+    # constant V -> constant O
+    w.v[:] = 0.75
+    o, st = run_attention(w)
+    assert st[0] == 0 and (o[0, :cfg.seq].float() - 0.75).abs().max().item() < 4e-3
+    # Q = 0 -> O is the mean of the selected V rows (uniform weights), LSE = log(#keys)
+    w.v.copy_(torch.stack([I.make_head_tensor(cfg, "v", 0)]).cuda())
+    w.q.zero_()
+    lse = torch.empty((1, cfg.seq), dtype=torch.float32, device="cuda")
+    o, st = run_attention(w, lse=lse)
+    V = w.head_f64("v", 0)
+    b = cfg.block
+    for i in (0, cfg.n_blocks // 2, cfg.n_blocks - 1):
+        keys = np.concatenate([np.arange(j * b, min((j + 1) * b, cfg.seq)) for j in np.nonzero(w.masks[0][i])[0]])
+        assert np.abs(o[0, i * b].float().cpu().numpy() - V[keys].mean(0)).max() < 4e-3
+        assert abs(lse[0, i * b].item() - math.log(len(keys))) < 1e-3
+    # large scores: the reference-max handling must not overflow
+    w.q.copy_(torch.stack([I.make_head_tensor(cfg, "q", 0)]).cuda())
+    o, st = run_attention(w, scale=4.0)
+    ref, _ = _oracle_head(w, 0, 4.0)
+    mx, mean = error_stats(o[0, :cfg.seq].float().cpu().numpy(), ref)
+    assert st[0] == 0 and np.isfinite(o[0, :cfg.seq].float().cpu().numpy()).all()
+    assert mx <= 4e-2 and mean <= MEAN_ABS     # near one-hot softmax: bf16 rounding of O dominates
+
+
+def _sample_tasks(nnz, rng, n_random=12):
+    m_b = len(nnz)
+    rows = {0, m_b - 1, int(np.argmin(nnz)), int(np.argmax(nnz))}
+    rows.update(int(r) for r in rng.choice(m_b, size=min(n_random, m_b), replace=False))
+    return sorted(rows)
+
+
+FULL = ["wan480p", "wan720p", "ltxmixed", "long720p"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_sampled_parity_and_invariance(name):
+    """BASELINE configs at full size, in the launch configuration the bench times: sampled
+    (head, row) tasks against the oracle; the whole output bitwise natural vs planned order."""
+    cfg = I.CONFIGS[name]
+    w = Workload(cfg)
+    W = wb.default_wave_size()
+    d = wb.plan_desc_default(heads=cfg.heads, n_q_blocks=cfg.n_blocks, n_kv_blocks=cfg.n_blocks, wave_size=W,
+                             mode=wb.FORCE_REORDER, seed=cfg.plan_seed)
+    plan = wb.plan_bitmap(d, w.bitmap)
+    nat, st = run_attention(w, out=torch.zeros_like(w.o))
+    assert st == [0, 0, 0, 0]
+    o, st = run_attention(w, row_order=plan.row_order)
+    assert st == [0, 0, 0, 0]
+    assert torch.equal(nat, o)
+    order = plan.row_order.cpu().numpy()
+    assert np.array_equal(np.sort(order, axis=1), np.tile(np.arange(cfg.n_blocks), (cfg.heads, 1)))
+    rng = np.random.default_rng(cfg.tensor_seed)
+    heads = sorted({0, cfg.heads - 1, *rng.choice(cfg.heads, size=2, replace=False).tolist()})
+    b = cfg.block
+    errs = []
+    for h in heads:
+        Q, K, V = (w.head_f64(x, h) for x in "qkv")
+        nnz = wo.row_nnz(w.masks[h])
+        for i in _sample_tasks(nnz, rng):
+            lo, hi = i * b, min((i + 1) * b, cfg.seq)
+            ref, _ = wo.attention_block_row(Q[lo:hi], K, V, np.nonzero(w.masks[h][i])[0], b, cfg.seq,
+                                            1 / math.sqrt(cfg.head_dim))
+            errs.append(error_stats(o[h, lo:hi].float().cpu().numpy(), ref))
+    assert max(e[0] for e in errs) <= MAX_ABS and max(e[1] for e in errs) <= MEAN_ABS
