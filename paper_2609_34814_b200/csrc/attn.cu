@@ -11,14 +11,17 @@
 // Structure of one CTA (320 threads):
 //   warp 0      producer: takes tickets, publishes tasks, issues TMA loads of the Q tile and
 //               of the K/V tiles (128-byte-swizzled slabs) into a shared-memory ring
-//   warp 1      MMA issuer: S = Q K^T and O += P V as tcgen05.mma with fp32 accumulators in
-//               tensor memory; S is double-buffered so that S_{j+1} is computed while the
-//               softmax of S_j runs
-//   warps 2-9   softmax: thread (row, column half) reads its half row of S from tensor
-//               memory, keeps the running max / sum, writes P (bf16) into shared memory in
-//               the operand layout of the second MMA, rescales O in tensor memory only when
-//               the max grew by more than 2^8, and finally normalises and stores O at the
-//               ORIGINAL row position (no inverse permutation pass)
+//   warp 1      MMA issuer: S = Q K^T (operands in shared memory) and O += P V (P read from
+//               tensor memory) as tcgen05.mma with fp32 accumulators in tensor memory
+//   warps 2-5   softmax group 0: the even-numbered blocks of the row's list
+//   warps 6-9   softmax group 1: the odd-numbered blocks
+//               Each group owns one S/P buffer and one partial output in tensor memory and
+//               its own running (max, sum): while one group runs the softmax of block j the
+//               tensor cores work for the other (P_{j-1} V_{j-1}, then Q K_{j+1}^T).  A thread
+//               owns one row: it reads S, writes P (bf16) over the same columns, and rescales
+//               its partial O only when the max grew by more than 2^8.  The epilogue merges
+//               the two partial results exactly, normalises and stores O at the ORIGINAL row
+//               position (no inverse permutation pass).
 // Every wait on an mbarrier is bounded; when one runs out the CTA records
 // {WAVEAL_ERR_TIMEOUT, site} and all roles leave through the common teardown.
 #include <cuda.h>
@@ -36,6 +39,20 @@ constexpr long long kTimeoutCycles = 4000000000ll;   // ~2 s at boost clock
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// One lane of a converged warp gets true.  tcgen05.mma / tcgen05.commit are issued under
+// this predicate, one instruction at a time, with their operands computed by the whole warp:
+// the operands then stay in uniform registers (a branch on the lane index instead makes the
+// compiler move every operand from vector registers, which halves the MMA issue rate).
+__device__ __forceinline__ uint32_t elect_one() {
+  uint32_t pred = 0;
+  asm volatile(
+      "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
+      "elect.sync rx|px, 0xFFFFFFFF;\n\t"
+      "@px mov.s32 %0, 1;\n\t}"
+      : "+r"(pred));
+  return pred;
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
@@ -50,6 +67,18 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// non-blocking probe (try_wait may suspend the thread for a while when the phase is not complete)
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -80,18 +109,31 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
+__device__ __forceinline__ void tc_commit(uint32_t bar) {   // whole warp calls; one lane issues
+  if (elect_one())
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate, one CTA
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  if (elect_one())
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]: A is 128 lanes x K bf16, two K elements per 32-bit column
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  if (elect_one())
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
@@ -132,9 +174,13 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       : "memory")
 
 __device__ __forceinline__ float ex2(float x) {
+#ifdef WAVEAL_DBG_NOEXP
+  return x * 0.001f + 0.5f;
+#else
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+#endif
 }
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -179,25 +225,40 @@ template <int BLOCK, int D>
 struct Geo {
   static constexpr int BQ = BLOCK, BK = BLOCK;
   static constexpr int SLABS = D / 64;               // 128-byte column slabs of a Q/K/V tile
-  static constexpr int PSLABS = BK / 64;             // slabs of the P tile (keys are its K dim)
-  static constexpr int Q_BYTES = SLABS * 128 * 128;  // smem reserved for 128 MMA rows
-  static constexpr int P_BYTES = PSLABS * 128 * 128;
+  static constexpr int Q_BYTES = SLABS * 128 * 128;  // smem reserved for the 128 MMA rows
   static constexpr int TILE_BYTES = SLABS * BK * 128;
   static constexpr int KV_SLAB_BYTES = BK * 128;
-  static constexpr int NSTAGE = BLOCK == 128 ? 4 : 8;
-  static constexpr int CS = BK / 2;                  // S columns per softmax thread
-  static constexpr int CO = D / 2;                   // O columns per softmax thread
+  static constexpr int NSTAGE_RAW = (200 * 1024 - Q_BYTES) / TILE_BYTES;
+  static constexpr int NSTAGE = NSTAGE_RAW > 8 ? 8 : NSTAGE_RAW;
+  static constexpr int PC = BK / 2;                  // tensor-memory columns of a P tile (bf16 pairs)
+  static constexpr int CO = D / 2;                   // O columns per epilogue thread
   static constexpr int OFF_Q = 0;
-  static constexpr int OFF_P = OFF_Q + Q_BYTES;
-  static constexpr int OFF_KV = OFF_P + P_BYTES;
+  static constexpr int OFF_KV = OFF_Q + Q_BYTES;
   static constexpr int OFF_BAR = OFF_KV + NSTAGE * TILE_BYTES;
-  static constexpr int N_BAR = 2 + 2 + 2 + 2 * NSTAGE + 2 + 2 + 2 + 1;
+  static constexpr int N_BAR = 4 + 2 + 2 * NSTAGE + 2 + 2 + 3;
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
-  static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
-  static constexpr int OFF_MISC = OFF_MX + 2 * 2 * 128 * 4;
+  static constexpr int OFF_EX = OFF_TASK + 2 * (int)sizeof(Task);
+  static constexpr int OFF_MISC = OFF_EX + 2 * 2 * 128 * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for 1024-byte alignment
-  static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL = 256, TMEM_COLS = 512;
+  // tensor memory: two S/P buffers (even / odd K/V blocks) and the two partial outputs
+  static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL0 = 256, O_COL1 = 384, TMEM_COLS = 512;
 };
+
+#ifdef WAVEAL_TRACE
+// debug build only: four tracer threads of CTA 0 append (tag, block, clock) records to their own
+// region after the 256-byte workspace header (plain stores, no atomics)
+#define TRACE_DECL int trace_n_ = 0
+#define TRACE(role, tag, j)                                                                    \
+  do {                                                                                         \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && trace_n_ < 4000) {                       \
+      int* r_ = p.ws + 64 + (role) * 8000 + 2 * trace_n_;                                      \
+      r_[0] = (tag) | ((j) << 8); r_[1] = (int)clock64(); ++trace_n_;                          \
+    }                                                                                          \
+  } while (0)
+#else
+#define TRACE_DECL
+#define TRACE(role, tag, j) do {} while (0)
+#endif
 
 struct Ctx {
   uint32_t bar_base;
@@ -234,6 +295,14 @@ __device__ __forceinline__ bool warp_wait(const Ctx& c, uint32_t bar, uint32_t p
   return __all_sync(0xffffffffu, mbar_wait(c, bar, parity, site));
 }
 
+// Second half of a split wait: `tok` is the answer of a non-blocking probe issued earlier (before the
+// preceding group of MMAs, so that its latency hides behind their issue: the tensor pipe's
+// queue is short, and any pause of the issuing warp between two MMAs starves it).
+__device__ __forceinline__ bool finish_wait(const Ctx& c, uint32_t bar, uint32_t parity, uint32_t tok, int site) {
+  if (__all_sync(0xffffffffu, tok)) return true;
+  return warp_wait(c, bar, parity, site);
+}
+
 template <int BLOCK, int D>
 __global__ void __launch_bounds__(kThreads, 1)
 k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -242,17 +311,17 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // provably warp-uniform role index
 
-  // barrier addresses
   const uint32_t bar0 = sbase + G::OFF_BAR;
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   constexpr int B_TASK_FULL = 0, B_TASK_EMPTY = 2, B_Q_FULL = 4, B_Q_EMPTY = 5, B_KV_FULL = 6,
-                B_KV_EMPTY = 6 + G::NSTAGE, B_S_FULL = 6 + 2 * G::NSTAGE, B_S_EMPTY = B_S_FULL + 2,
-                B_P_FULL = B_S_EMPTY + 2, B_PV_DONE = B_P_FULL + 1, B_FINAL = B_PV_DONE + 1;
+                B_KV_EMPTY = 6 + G::NSTAGE, B_S_FULL = 6 + 2 * G::NSTAGE, B_P_FULL = B_S_FULL + 2,
+                B_O_FULL = B_P_FULL + 2, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1;
   static_assert(B_FINAL + 1 <= G::N_BAR, "barrier count");
   Task* tasks = reinterpret_cast<Task*>(smem + G::OFF_TASK);
-  float* mx = reinterpret_cast<float*>(smem + G::OFF_MX);            // [2][2][128]
+  float2* ex = reinterpret_cast<float2*>(smem + G::OFF_EX);          // [task parity][group][128] (m, l)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + G::OFF_MISC);
   volatile int* abort_smem = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 4);
   Ctx ctx{bar0, abort_smem, p.ws, p.dev_status};
@@ -262,9 +331,9 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     mbar_init(BAR(B_Q_FULL), 1);
     mbar_init(BAR(B_Q_EMPTY), 1);
     for (int i = 0; i < G::NSTAGE; ++i) { mbar_init(BAR(B_KV_FULL + i), 1); mbar_init(BAR(B_KV_EMPTY + i), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_S_FULL + i), 1); mbar_init(BAR(B_S_EMPTY + i), 8); }
-    mbar_init(BAR(B_P_FULL), 8);
-    mbar_init(BAR(B_PV_DONE), 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_S_FULL + i), 1); mbar_init(BAR(B_P_FULL + i), 4); }
+    mbar_init(BAR(B_O_FULL), 1);
+    mbar_init(BAR(B_O_FREE), 8);
     mbar_init(BAR(B_FINAL), 1);
     *abort_smem = 0;
     fence_mbar_init();
@@ -286,14 +355,13 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     // ============================================================== producer
     if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); }
     uint32_t task_it = 0, q_it = 0, kv_it = 0;
+    TRACE_DECL;
     bool ok = true;
-    uint32_t armed_mask = 0, armed_parity = 0;   // per-stage: a load is (or was) in flight with this parity
+    uint32_t armed_mask = 0, armed_parity = 0;   // per stage: parity of the last load armed on it
     bool q_armed = false; uint32_t q_armed_parity = 0;
     while (ok) {
       long long t = 0;
-      if (lane == 0) {
-        t = (p.ws[1] != 0) ? p.total_tasks : (long long)(unsigned)atomicAdd(&p.ws[0], 1);
-      }
+      if (lane == 0) t = (p.ws[1] != 0) ? p.total_tasks : (long long)(unsigned)atomicAdd(&p.ws[0], 1);
       t = __shfl_sync(0xffffffffu, t, 0);
       Task tk{};
       if (t >= p.total_tasks) {
@@ -330,38 +398,42 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
       q_armed = true; q_armed_parity = q_it & 1;
       ++q_it;
-      // K/V tiles in consumption order: K_0, then for each j: K_{j+1} (if any), V_j
-      const int n_tiles = 2 * tk.n;
-      int chunk_base = -32, my_idx = 0;
-      for (int e = 0; e < n_tiles && ok; ++e) {
-        // tile e: e == 0 -> K_0; odd e -> (e+1)/2 < n ? K_{(e+1)/2} : V_{n-1}...
-        // sequence: K0, K1, V0, K2, V1, ..., K_{n-1}, V_{n-2}, V_{n-1}
-        int j; bool is_k;
-        if (e == 0) { j = 0; is_k = true; }
-        else if (e == n_tiles - 1) { j = tk.n - 1; is_k = false; }
-        else if (e & 1) { j = (e + 1) / 2; is_k = true; }
-        else { j = e / 2 - 1; is_k = false; }
+      // K/V tiles in the order the MMA warp consumes them: K_0, K_1, then V_j, K_{j+2} for each j
+      int chunk_base = -64, my_idx = 0;
+      auto load_tile = [&](bool is_k, int j) -> bool {
         if (j < chunk_base || j >= chunk_base + 32) {
           chunk_base = j & ~31;
-          int q = chunk_base + lane;
+          const int q = chunk_base + lane;
           my_idx = q < tk.n ? p.kv_idx[tk.lo + q] : 0;
         }
         int blk = __shfl_sync(0xffffffffu, my_idx, j - chunk_base);
         if (blk < 0 || blk >= p.n_b) blk = 0;            // malformed list: stay in range
         const uint32_t st = kv_it % G::NSTAGE, sph = (kv_it / G::NSTAGE) & 1;
-        ok = warp_wait(ctx, BAR(B_KV_EMPTY + st), sph ^ 1, 3);
-        if (!ok) break;
+        if (!warp_wait(ctx, BAR(B_KV_EMPTY + st), sph ^ 1, 3)) return false;
+        TRACE(3, 20 + (is_k ? 0 : 1), j);
         if (lane == 0) {
+#ifdef WAVEAL_DBG_NOLOAD
+          if (kv_it >= (uint32_t)G::NSTAGE) { mbar_arrive(BAR(B_KV_FULL + st)); } else
+#endif
+          {
           mbar_expect_tx(BAR(B_KV_FULL + st), G::TILE_BYTES);
           const CUtensorMap* tm = is_k ? &tmK : &tmV;
 #pragma unroll
           for (int s = 0; s < G::SLABS; ++s)
             tma_load_3d(sbase + G::OFF_KV + st * G::TILE_BYTES + s * G::KV_SLAB_BYTES, tm, s * 64, blk * G::BK, tk.h,
                         BAR(B_KV_FULL + st));
+          }
         }
         armed_mask |= 1u << st;
         armed_parity = (armed_parity & ~(1u << st)) | (sph << st);
         ++kv_it;
+        return true;
+      };
+      ok = load_tile(true, 0);
+      if (ok && tk.n > 1) ok = load_tile(true, 1);
+      for (int j = 0; j < tk.n && ok; ++j) {
+        ok = load_tile(false, j);
+        if (ok && j + 2 < tk.n) ok = load_tile(true, j + 2);
       }
     }
     if (*abort_smem) {
@@ -378,80 +450,132 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
   } else if (warp == 1) {
     // ============================================================== MMA issuer
+    // Every operand of a tcgen05 instruction (descriptors, tensor-memory addresses, barrier
+    // addresses) must stay warp-uniform in the compiler's eyes, otherwise each MMA pays for
+    // moves into uniform registers and the issue rate drops below the tensor pipe's: values
+    // read from shared memory are broadcast with a shuffle, ring positions are advanced by
+    // compare-and-reset instead of modulo.
     constexpr uint32_t IDESC_QK = make_idesc(128, G::BK, false);
     constexpr uint32_t IDESC_PV = make_idesc(128, D, true);
-    uint32_t task_it = 0, q_it = 0, kv_it = 0, s_it = 0, p_it = 0;
+    uint32_t task_slot = 0, task_ph = 0, q_ph = 0, o_ph = 1, kv_st = 0, kv_ph = 0;
+    uint32_t p_ph0 = 0, p_ph1 = 0;
+    TRACE_DECL;
+    const uint64_t qdesc0 = make_desc(sbase + G::OFF_Q, 16, 1024);
+    const uint64_t kdesc0 = make_desc(sbase + G::OFF_KV, 16, 1024);
+    const uint64_t vdesc0 = make_desc(sbase + G::OFF_KV, G::KV_SLAB_BYTES, 1024);
     bool ok = true;
     while (ok) {
-      const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
-      ok = warp_wait(ctx, BAR(B_TASK_FULL + slot), ph, 10);
+      ok = warp_wait(ctx, BAR(B_TASK_FULL + task_slot), task_ph, 10);
       if (!ok) break;
-      const int n = tasks[slot].n;
+      const int n = __shfl_sync(0xffffffffu, tasks[task_slot].n, 0);
       __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + slot));
-      ++task_it;
+      if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + task_slot));
+      task_slot ^= 1;
+      task_ph ^= (task_slot == 0);
       if (n < 0) break;
       if (n == 0) continue;
-      ok = warp_wait(ctx, BAR(B_Q_FULL), q_it & 1, 11);
+      ok = warp_wait(ctx, BAR(B_Q_FULL), q_ph, 11);
       if (!ok) break;
-      ++q_it;
-      // one QK^T: S[buf] = Q K_j^T
-      auto issue_qk = [&]() -> bool {
-        const uint32_t st = kv_it % G::NSTAGE, sph = (kv_it / G::NSTAGE) & 1;
-        const uint32_t buf = s_it & 1, bph = (s_it >> 1) & 1;
-        if (!warp_wait(ctx, BAR(B_KV_FULL + st), sph, 12)) return false;
-        if (!warp_wait(ctx, BAR(B_S_EMPTY + buf), bph ^ 1, 13)) return false;
-        tc_fence_after();
-        if (lane == 0) {
-          const uint32_t kbase = sbase + G::OFF_KV + st * G::TILE_BYTES;
+      q_ph ^= 1;
+      // S[g] = Q K_j^T (g = j & 1); overwrites the P tile that aliases S[g], which the
+      // preceding P V of the same parity (issued earlier by this warp) has consumed.
+      // The caller has already waited for the K tile in stage kv_st.
+      auto issue_qk = [&](uint32_t g) {
+        TRACE(0, 4, (int)kv_st);
+        {
+          // descriptors differ from the per-kernel bases only in the 14-bit address field
+          const uint64_t kd = kdesc0 + (uint64_t)(kv_st * (uint32_t)(G::TILE_BYTES >> 4));
+          const uint32_t d_s = tmem_base + g * 128u;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
-            uint64_t a = make_desc(sbase + G::OFF_Q + (k / 4) * 128 * 128 + (k % 4) * 32, 16, 1024);
-            uint64_t b = make_desc(kbase + (k / 4) * G::KV_SLAB_BYTES + (k % 4) * 32, 16, 1024);
-            umma_bf16(tmem_base + (buf ? G::S_COL1 : G::S_COL0), a, b, IDESC_QK, k > 0);
+#ifndef WAVEAL_DBG_SKIP_QK
+            umma_bf16(d_s, qdesc0 + (uint64_t)(((k / 4) * 128 * 128 + (k % 4) * 32) >> 4),
+                      kd + (uint64_t)(((k / 4) * G::KV_SLAB_BYTES + (k % 4) * 32) >> 4), IDESC_QK, k > 0);
+#endif
           }
-          tc_commit(BAR(B_KV_EMPTY + st));
-          tc_commit(BAR(B_S_FULL + buf));
+          tc_commit(BAR(B_KV_EMPTY + kv_st));
+          tc_commit(BAR(B_S_FULL + g));
         }
-        __syncwarp();
-        ++kv_it; ++s_it;
-        return true;
+        TRACE(0, 5, (int)kv_st);
+        if (++kv_st == (uint32_t)G::NSTAGE) { kv_st = 0; kv_ph ^= 1; }
       };
-      ok = issue_qk();
-      // once the last QK^T of the task is issued, its completion frees the Q tile
-      if (ok && n == 1) { if (lane == 0) tc_commit(BAR(B_Q_EMPTY)); __syncwarp(); }
+      ok = warp_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, 12);
+      if (!ok) break;
+      issue_qk(0);
+      if (n > 1) {
+        ok = warp_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, 12);
+        if (!ok) break;
+        issue_qk(1);
+      }
+      if (n <= 2) tc_commit(BAR(B_Q_EMPTY));
+      // the partial outputs of the previous task have been read by the epilogue
+      ok = warp_wait(ctx, BAR(B_O_FREE), o_ph, 16);
+      if (!ok) break;
+      o_ph ^= 1;
+      // answers for the first P V of the task
+      uint32_t tok_p = mbar_test_wait(BAR(B_P_FULL + 0), p_ph0);
+      uint32_t tok_v = mbar_test_wait(BAR(B_KV_FULL + kv_st), kv_ph);
       for (int j = 0; j < n && ok; ++j) {
-        if (j + 1 < n) {
-          ok = issue_qk();
-          if (!ok) break;
-          if (j + 2 == n) { if (lane == 0) tc_commit(BAR(B_Q_EMPTY)); __syncwarp(); }
-        }
-        // O (+)= P_j V_j
-        const uint32_t st = kv_it % G::NSTAGE, sph = (kv_it / G::NSTAGE) & 1;
-        ok = warp_wait(ctx, BAR(B_P_FULL), p_it & 1, 14);
+        const uint32_t g = (uint32_t)j & 1u;
+        // O[g] (+)= P_j V_j, P_j read from tensor memory
+        ok = finish_wait(ctx, BAR(B_P_FULL + g), g ? p_ph1 : p_ph0, tok_p, 14);
         if (!ok) break;
-        ok = warp_wait(ctx, BAR(B_KV_FULL + st), sph, 15);
+        if (g) p_ph1 ^= 1; else p_ph0 ^= 1;
+        TRACE(0, 1, j);
+        ok = finish_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, tok_v, 15);
         if (!ok) break;
+        TRACE(0, 2, j);
+        const bool more_qk = j + 2 < n;
+        // the K tile of block j+2 sits in the stage after this V tile: ask now, use after the MMAs
+        uint32_t k_st = kv_st + 1, k_ph = kv_ph;
+        if (k_st == (uint32_t)G::NSTAGE) { k_st = 0; k_ph ^= 1; }
+        uint32_t tok_k = more_qk ? mbar_test_wait(BAR(B_KV_FULL + k_st), k_ph) : 1u;
         tc_fence_after();
-        if (lane == 0) {
-          const uint32_t vbase = sbase + G::OFF_KV + st * G::TILE_BYTES;
+        {
+          // V tile as the N x K operand with N (head_dim) contiguous: 8 keys per 1024-byte
+          // group along K (16 keys = 2048 bytes per MMA), next 64 columns of head_dim one slab further
+          const uint64_t vd = vdesc0 + (uint64_t)(kv_st * (uint32_t)(G::TILE_BYTES >> 4));
+          const uint32_t pbase = tmem_base + g * 128u;
+          const uint32_t d_o = tmem_base + G::O_COL0 + g * 128u;
+          if (j >= 2) {
 #pragma unroll
-          for (int k = 0; k < G::BK / 16; ++k) {
-            uint64_t a = make_desc(sbase + G::OFF_P + (k / 4) * 128 * 128 + (k % 4) * 32, 16, 1024);
-            // V tile as the N x K operand with N (head_dim) contiguous: 8 keys per 1024-byte
-            // group along K, next 64 columns of head_dim one slab further
-            uint64_t b = make_desc(vbase + k * 16 * 128, G::KV_SLAB_BYTES, 1024);
-            umma_bf16(tmem_base + G::O_COL, a, b, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < G::BK / 16; ++k) {
+#ifndef WAVEAL_DBG_SKIP_PV
+              umma_bf16_ts(d_o, pbase + k * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, 1u);
+#endif
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < G::BK / 16; ++k) {
+#ifndef WAVEAL_DBG_SKIP_PV
+              umma_bf16_ts(d_o, pbase + k * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, k > 0 ? 1u : 0u);
+#endif
+            }
           }
-          tc_commit(BAR(B_KV_EMPTY + st));
-          tc_commit(BAR(B_PV_DONE));
+          tc_commit(BAR(B_KV_EMPTY + kv_st));
+          if (j == n - 1) tc_commit(BAR(B_O_FULL));
         }
-        __syncwarp();
-        ++kv_it; ++p_it;
+        TRACE(0, 3, j);
+        if (++kv_st == (uint32_t)G::NSTAGE) { kv_st = 0; kv_ph ^= 1; }
+        if (more_qk) {
+          ok = finish_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, tok_k, 12);
+          if (!ok) break;
+        }
+        // answers for the next P V (other group's P tile; its V tile follows the K tile just checked)
+        if (j + 1 < n) {
+          uint32_t v_st = kv_st, v_ph = kv_ph;
+          if (more_qk) { if (++v_st == (uint32_t)G::NSTAGE) { v_st = 0; v_ph ^= 1; } }
+          tok_p = mbar_test_wait(BAR(B_P_FULL + (g ^ 1u)), g ? p_ph0 : p_ph1);
+          tok_v = mbar_test_wait(BAR(B_KV_FULL + v_st), v_ph);
+        }
+        if (more_qk) {
+          issue_qk(g);
+          if (j + 2 == n - 1) tc_commit(BAR(B_Q_EMPTY));
+        }
       }
     }
-    // every MMA issued by this thread has completed before tensor memory is released
-    if (lane == 0) tc_commit(BAR(B_FINAL));
+    // every MMA issued by this warp has completed before tensor memory is released
+    tc_commit(BAR(B_FINAL));
     __syncwarp();
     {
       long long t0 = clock64();
@@ -459,12 +583,16 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
   } else {
     // ============================================================== softmax / epilogue
-    const int sw = warp - kSoftmaxWarp0;       // 0..7
+    // group 0 (warps 2-5) takes the even K/V blocks of a row's list, group 1 (warps 6-9) the
+    // odd ones; each keeps its own reference max, sum and partial output; the epilogue merges.
+    const int g = (warp - kSoftmaxWarp0) >> 2;
     const int quad = warp & 3;                 // tensor-memory lane quadrant this warp may access
-    const int half = sw >> 2;                  // which half of the S / O columns
     const int r = quad * 32 + lane;            // row of the 128-row MMA tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    uint32_t task_it = 0, s_it = 0, pv_it = 0;
+    const uint32_t s_addr = tmem_base + lane_addr + (g ? G::S_COL1 : G::S_COL0);
+    const uint32_t o_own = tmem_base + lane_addr + (g ? G::O_COL1 : G::O_COL0);
+    uint32_t task_it = 0, s_it = 0, o_it = 0;
+    TRACE_DECL;
     bool ok = true;
     while (ok) {
       const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
@@ -473,49 +601,58 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const Task tk = tasks[slot];
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + slot));
+      float2* exb = ex + (task_it & 1) * 256;
       ++task_it;
       if (tk.n < 0) break;
       const long long q_tok = (long long)tk.row * G::BQ + r;
       const bool row_live = r < G::BQ && q_tok < p.seq_q;
-      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + half * G::CO;
+      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + g * G::CO;
       if (tk.n == 0) {
         if (row_live) {
 #pragma unroll
           for (int c = 0; c < G::CO / 8; ++c) reinterpret_cast<uint4*>(o_ptr)[c] = make_uint4(0, 0, 0, 0);
-          if (p.lse && half == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
+          if (p.lse && g == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
         }
         continue;
       }
       float m_used = -INFINITY, l_run = 0.f;
-      for (int j = 0; j < tk.n && ok; ++j) {
-        const uint32_t buf = s_it & 1, bph = (s_it >> 1) & 1;
-        ok = warp_wait(ctx, BAR(B_S_FULL + buf), bph, 21);
+      for (int j = g; j < tk.n && ok; j += 2) {
+        ok = warp_wait(ctx, BAR(B_S_FULL + g), s_it & 1, 21);
         if (!ok) break;
+        ++s_it;
+        if (quad == 2) TRACE(1 + g, 10 + g, j);
         tc_fence_after();
-        uint32_t sv[G::CS];
-        const uint32_t s_addr = tmem_base + lane_addr + (buf ? G::S_COL1 : G::S_COL0) + half * G::CS;
-#pragma unroll
-        for (int c = 0; c < G::CS; c += 32) WAVEAL_TMEM_LD32(s_addr + c, sv, c);
-#pragma unroll
-        for (int c = 0; c < G::CS; c += 32) WAVEAL_TMEM_WAIT_LD32(sv, c);
+#ifdef WAVEAL_DBG_NOSOFTMAX
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_S_EMPTY + buf));
-        ++s_it;
+        if (lane == 0) mbar_arrive(BAR(B_P_FULL + g));
+        continue;
+#endif
+        uint32_t sv[G::BK];
+#pragma unroll
+        for (int c = 0; c < G::BK; c += 32) WAVEAL_TMEM_LD32(s_addr + c, sv, c);
+#pragma unroll
+        for (int c = 0; c < G::BK; c += 32) WAVEAL_TMEM_WAIT_LD32(sv, c);
+        if (quad == 2) TRACE(1 + g, 12 + g, j);
         // scores of keys beyond seq_kv (ragged last block) do not exist
         if (j == tk.n - 1 && tk.tail_valid < G::BK) {
 #pragma unroll
-          for (int c = 0; c < G::CS; ++c)
-            if (half * G::CS + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
+          for (int c = 0; c < G::BK; ++c)
+            if (c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
         }
-        float mloc = -INFINITY;
+        // row max with eight independent chains (a single chain of 128 dependent max ops
+        // would cost more than the exponentials)
+        float mx8[8];
 #pragma unroll
-        for (int c = 0; c < G::CS; ++c) mloc = fmaxf(mloc, __uint_as_float(sv[c]));
-        float* mxb = mx + (j & 1) * 256;
-        mxb[half * 128 + r] = mloc;
-        named_bar_sync(1 + quad, 64);
-        const float m_blk = fmaxf(mloc, mxb[(half ^ 1) * 128 + r]) * p.sl2;
-        const float m_cand = fmaxf(m_used, m_blk);
+        for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(sv[i]);
+#pragma unroll
+        for (int c = 8; c < G::BK; c += 8) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(sv[c + i]));
+        }
+        const float mloc = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                                 fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+        const float m_cand = fmaxf(m_used, mloc * p.sl2);
         // keep the stale reference max unless it is exceeded by more than 2^8 (exact: the
         // final normalisation divides by a sum taken with the same reference)
         const bool grow = __any_sync(0xffffffffu, m_cand > m_used + 8.0f);
@@ -525,89 +662,94 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           m_used = m_cand;
           l_run *= alpha;
         }
-        uint32_t pk[G::CS / 2];
-        float lsum = 0.f;
-        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+        uint32_t pk[G::PC];
+        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+        // p' = 2^(s*scale*log2e - m + log2(1 + 2^-9)); P is p' cut to its top 16 bits (one byte
+        // permute per pair instead of a conversion on the transcendental pipe).  The extra
+        // factor centres the cut's error around zero, and the row sum adds the SAME cut values
+        // the tensor core multiplies with, so numerator and denominator stay consistent.
+        const float neg_m = ((m_used == -INFINITY) ? 0.f : -m_used) + 0.0028150156f;
 #pragma unroll
-        for (int c = 0; c < G::CS; c += 2) {
-          float p0 = ex2(fmaf(__uint_as_float(sv[c]), p.sl2, neg_m));
-          float p1 = ex2(fmaf(__uint_as_float(sv[c + 1]), p.sl2, neg_m));
-          lsum += p0 + p1;
-          __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-          pk[c / 2] = *reinterpret_cast<uint32_t*>(&b2);
+        for (int c = 0; c < G::BK; c += 2) {
+          const uint32_t b0 = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c]), p.sl2, neg_m)));
+          const uint32_t b1 = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c + 1]), p.sl2, neg_m)));
+          ls4[(c >> 1) & 3] += __uint_as_float(b0 & 0xFFFF0000u) + __uint_as_float(b1 & 0xFFFF0000u);
+          pk[c / 2] = __byte_perm(b0, b1, 0x7632);
         }
+        const float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
         l_run += lsum;
-        // P_{j-1} V_{j-1} must be complete before O is rescaled or the P tile is overwritten
-        if (j > 0) {
-          ok = warp_wait(ctx, BAR(B_PV_DONE), pv_it & 1, 22);
-          if (!ok) break;
-          ++pv_it;
-          tc_fence_after();
-          if (grow) {
-            uint32_t ov[G::CO];
-            const uint32_t o_addr = tmem_base + lane_addr + G::O_COL + half * G::CO;
+        if (quad == 2) TRACE(1 + g, 14 + g, j);
+        // P_j (bf16 pairs) over the first half of the columns of S[g]
 #pragma unroll
-            for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(o_addr + c, ov, c);
+        for (int c = 0; c < G::PC; c += 32) WAVEAL_TMEM_ST32(s_addr + c, pk, c);
+        // S_FULL of block j implies that P V of block j-2 is complete: O[g] may be rescaled
+        if (grow && j >= 2) {
 #pragma unroll
-            for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(ov, c);
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t ov[32];
+            WAVEAL_TMEM_LD32(o_own + c0, ov, 0);
+            WAVEAL_TMEM_WAIT_LD32(ov, 0);
 #pragma unroll
-            for (int c = 0; c < G::CO; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-#pragma unroll
-            for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_ST32(o_addr + c, ov, c);
-            tc_wait_st();
+            for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+            WAVEAL_TMEM_ST32(o_own + c0, ov, 0);
           }
         }
-        // P tile, K-major with 128-byte swizzle: key k of row r lives in slab k/64 at
-        // r*128 + ((k%64)/8 ^ (r%8))*16 + (k%8)*2
-        {
-          unsigned char* prow = smem + G::OFF_P + r * 128;
-#pragma unroll
-          for (int c8 = 0; c8 < G::CS / 8; ++c8) {
-            const int k0 = half * G::CS + c8 * 8;
-            const int slab = k0 >> 6, chunk = (k0 & 63) >> 3;
-            uint4 v = make_uint4(pk[c8 * 4 + 0], pk[c8 * 4 + 1], pk[c8 * 4 + 2], pk[c8 * 4 + 3]);
-            *reinterpret_cast<uint4*>(prow + slab * 128 * 128 + ((chunk ^ (r & 7)) << 4)) = v;
-          }
-        }
-        fence_proxy_async();
+        tc_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_P_FULL));
+        if (lane == 0) mbar_arrive(BAR(B_P_FULL + g));
+        if (quad == 2) TRACE(1 + g, 16 + g, j);
       }
       if (!ok) break;
-      // ---- epilogue: O / l at the original row position
-      ok = warp_wait(ctx, BAR(B_PV_DONE), pv_it & 1, 23);
+      // ---- epilogue: merge the two partial results, normalise, store at the original rows
+      ok = warp_wait(ctx, BAR(B_O_FULL), o_it & 1, 23);
       if (!ok) break;
-      ++pv_it;
+      ++o_it;
       tc_fence_after();
-      float* lx = mx + (tk.n & 1) * 256;      // the buffer the last block did not use
-      lx[half * 128 + r] = l_run;
+      if (quad == 2) TRACE(1 + g, 18 + g, tk.n);
+      exb[g * 128 + r] = make_float2(m_used, l_run);
       named_bar_sync(1 + quad, 64);
-      const float l_tot = l_run + lx[(half ^ 1) * 128 + r];
+      const float2 oth = exb[(g ^ 1) * 128 + r];
+      const float m_all = fmaxf(m_used, oth.x);
+      const float a_self = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_all);
+      const float a_oth = (oth.x == -INFINITY) ? 0.f : ex2(oth.x - m_all);
+      const float l_tot = a_self * l_run + a_oth * oth.y;
       const float inv_l = 1.0f / l_tot;
-      uint32_t ov[G::CO];
-      const uint32_t o_addr = tmem_base + lane_addr + G::O_COL + half * G::CO;
+      const float w_e = (g == 0 ? a_self : a_oth) * inv_l, w_o = (g == 0 ? a_oth : a_self) * inv_l;
+      uint32_t oe[G::CO], oo[G::CO];
+      const uint32_t col0 = tmem_base + lane_addr + g * G::CO;
 #pragma unroll
-      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(o_addr + c, ov, c);
+      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(col0 + G::O_COL0 + c, oe, c);
+      if (tk.n >= 2) {
 #pragma unroll
-      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(ov, c);
+        for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(col0 + G::O_COL1 + c, oo, c);
+#pragma unroll
+        for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(oo, c);
+      } else {
+#pragma unroll
+        for (int c = 0; c < G::CO; ++c) oo[c] = 0u;
+      }
+#pragma unroll
+      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(oe, c);
       tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_O_FREE));
+      if (quad == 2) TRACE(1 + g, 30 + g, tk.n);
       if (row_live) {
 #pragma unroll
         for (int c = 0; c < G::CO; c += 8) {
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(ov[c + 2 * e]) * inv_l,
-                                                      __uint_as_float(ov[c + 2 * e + 1]) * inv_l);
+            float x0 = __uint_as_float(oe[c + 2 * e]) * w_e + __uint_as_float(oo[c + 2 * e]) * w_o;
+            float x1 = __uint_as_float(oe[c + 2 * e + 1]) * w_e + __uint_as_float(oo[c + 2 * e + 1]) * w_o;
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(x0, x1);
             w[e] = *reinterpret_cast<uint32_t*>(&b2);
           }
           *reinterpret_cast<uint4*>(o_ptr + c) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (p.lse && half == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_used + log2f(l_tot)) * 0.6931471805599453f;
+        if (p.lse && g == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_all + log2f(l_tot)) * 0.6931471805599453f;
       }
-      // the exchange buffer is reused by the next task's first block: keep the pair in step
-      named_bar_sync(1 + quad, 64);
     }
   }
 
@@ -682,7 +824,7 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   if ((s = make_map(&tk, K, D, d->seq_kv, d->heads, d->k_stride[0], d->k_stride[1], BLOCK, "K")) != WAVEAL_OK) return s;
   if ((s = make_map(&tv, V, D, d->seq_kv, d->heads, d->v_stride[0], d->v_stride[1], BLOCK, "V")) != WAVEAL_OK) return s;
   WAVEAL_CUDA_OK(cudaFuncSetAttribute(k_bsattn_fwd<BLOCK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES));
-  WAVEAL_CUDA_OK(cudaMemsetAsync(p.ws, 0, 16, st));
+  WAVEAL_CUDA_OK(cudaMemsetAsync(p.ws, 0, 16, st));  // ticket counter, abort flag (and the debug trace count)
   long long grid = p.total_tasks < sms ? p.total_tasks : sms;
   k_bsattn_fwd<BLOCK, D><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
   WAVEAL_CUDA_OK(cudaGetLastError());
