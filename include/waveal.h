@@ -126,6 +126,29 @@ waveal_status waveal_bitmap_to_csr(int32_t heads, int32_t n_q_blocks, int32_t n_
                                    int32_t* kv_block_indices_out /*dev or NULL*/, int64_t capacity,
                                    void* ws /*dev*/, size_t ws_bytes, void* cuda_stream);
 
+/* Same conversion for callers that have no way to provide a workspace: a plug-in that sits
+ * inside a serving engine between mask construction and the attention backend is handed
+ * tensors, not an allocator; the engine has planned all device memory up front, and a
+ * cudaMalloc / cudaFree in the middle of a denoising loop would stall every stream of the
+ * device.  This entry point therefore calls no allocation routine of CUDA or of any library:
+ * its scratch (the per-row counts) is a 1 MiB array built into the library image, which every
+ * GPU that loads the library holds until the process exits.
+ * (The paper has no counterpart of this call; it is a convenience of this library.)
+ *   - limit: heads * n_q_blocks <= waveal_noalloc_max_rows() (262,143); larger problems are
+ *     refused with WAVEAL_ERR_UNSUPPORTED before anything is enqueued;
+ *   - the first call on each device looks up the array's device address (with that device
+ *     current); make that first call before any stream capture begins;
+ *   - all calls share the one array: two calls whose kernels overlap on the GPU (different
+ *     streams, or different host threads) race and corrupt each other's row pointers; calls
+ *     enqueued on one stream are safe.  Nothing in the array has to be cleared between calls.
+ * Inputs and outputs are as for waveal_bitmap_to_csr and stay caller-owned. */
+waveal_status waveal_bitmap_to_csr_noalloc(int32_t heads, int32_t n_q_blocks, int32_t n_kv_blocks,
+                                           const uint64_t* mask_bits /*dev*/, int32_t* kv_row_ptr_out /*dev*/,
+                                           int32_t* kv_block_indices_out /*dev or NULL*/, int64_t capacity,
+                                           void* cuda_stream);
+/* Largest heads * n_q_blocks the call above accepts.  Host-only. */
+size_t waveal_noalloc_max_rows(void);
+
 typedef struct waveal_attn_desc {
   int32_t heads;            /* batch*heads; K/V heads == Q heads                              */
   int32_t seq_q, seq_kv;    /* true (unpadded) lengths                                        */

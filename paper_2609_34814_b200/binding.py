@@ -19,7 +19,8 @@ AUTO, FORCE_REORDER, FORCE_NATURAL, STAGE1_ONLY, STAGE2_ONLY = range(5)
 FLAG_SKIPPED, FLAG_SHORT_SEQ, FLAG_TOO_SPARSE, FLAG_ALREADY_LOCAL = 1, 2, 4, 8
 
 EXPORTS = ["waveal_plan_desc_default", "waveal_plan_workspace_bytes", "waveal_plan_bitmap", "waveal_plan_csr",
-           "waveal_bitmap_to_csr", "waveal_bsattn_workspace_bytes", "waveal_bsattn_fwd",
+           "waveal_bitmap_to_csr", "waveal_bitmap_to_csr_noalloc", "waveal_noalloc_max_rows",
+           "waveal_bsattn_workspace_bytes", "waveal_bsattn_fwd",
            "waveal_default_wave_size", "waveal_last_launch_count", "waveal_status_string", "waveal_last_error"]
 
 
@@ -69,6 +70,9 @@ def load() -> ctypes.CDLL:
         lib.waveal_plan_bitmap.argtypes = [ctypes.POINTER(PlanDesc), P, P, ctypes.c_size_t, ctypes.POINTER(PlanOut), P]
         lib.waveal_plan_csr.argtypes = [ctypes.POINTER(PlanDesc), P, P, P, ctypes.c_size_t, ctypes.POINTER(PlanOut), P]
         lib.waveal_bitmap_to_csr.argtypes = [I32, I32, I32, P, P, P, I64, P, ctypes.c_size_t, P]
+        lib.waveal_bitmap_to_csr_noalloc.argtypes = [I32, I32, I32, P, P, P, I64, P]
+        lib.waveal_bitmap_to_csr_noalloc.restype = ctypes.c_int
+        lib.waveal_noalloc_max_rows.restype = ctypes.c_size_t
         lib.waveal_bsattn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), ctypes.POINTER(ctypes.c_size_t)]
         lib.waveal_bsattn_fwd.argtypes = [ctypes.POINTER(AttnDesc), P, P, P, P, P, P, P, P, ctypes.c_float, P,
                                           ctypes.c_size_t, P, P]
@@ -199,6 +203,22 @@ def bitmap_to_csr(mask_bits, n_kv_blocks: int, capacity: Optional[int] = None, s
     _check(lib.waveal_bitmap_to_csr(H, M, n_kv_blocks, _ptr(mask_bits), _ptr(ptr), _ptr(idx), capacity, _ptr(ws),
                                     ws.numel(), _stream(stream)))
     return ptr, idx[:capacity]
+
+
+def noalloc_max_rows() -> int:
+    return int(load().waveal_noalloc_max_rows())
+
+
+def bitmap_to_csr_noalloc(mask_bits, n_kv_blocks: int, kv_row_ptr, kv_block_indices, stream=None):
+    """waveal_bitmap_to_csr_noalloc: for callers that cannot allocate device memory (an engine
+    plug-in handed pre-planned tensors).  Every buffer is the caller's: `kv_row_ptr` int32
+    [heads*M_B + 1] and `kv_block_indices` int32 [capacity] (or None for row pointers only)
+    are filled on the stream; the call itself allocates nothing, here or in the library, and
+    refuses problems with more than noalloc_max_rows() query-block rows."""
+    H, M, _ = mask_bits.shape
+    cap = 0 if kv_block_indices is None else kv_block_indices.numel()
+    _check(load().waveal_bitmap_to_csr_noalloc(H, M, n_kv_blocks, _ptr(mask_bits), _ptr(kv_row_ptr),
+                                               _ptr(kv_block_indices), cap, _stream(stream)))
 
 
 def attn_desc(q, k, v, o, seq_q: int, seq_kv: int, block: int, interleaved: bool = False) -> AttnDesc:

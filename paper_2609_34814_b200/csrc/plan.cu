@@ -15,6 +15,7 @@
 #include <cfloat>
 #include <climits>
 #include <cmath>
+#include <mutex>
 #include "host_common.h"
 
 namespace {
@@ -680,4 +681,58 @@ extern "C" waveal_status waveal_bitmap_to_csr(int32_t heads, int32_t n_q_blocks,
   WAVEAL_CUDA_OK(cudaGetLastError());
   waveal::launch_counter() = launches;
   return WAVEAL_OK;
+}
+
+// ------------------------------------------------------------------ entry point that allocates nothing
+
+// Scratch for waveal_bitmap_to_csr_noalloc: lives in the library image, so every GPU that
+// loads the library holds this 1 MiB until the process exits.
+#define WAVEAL_NOALLOC_SCRATCH_BYTES (1u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[WAVEAL_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mu;
+void* g_scratch_addr[kMaxDevices] = {};   // device address of g_noalloc_scratch, per device
+
+// In host code the array's name is only a handle; the address a kernel can use has to be
+// asked for, once per device, with that device current.
+waveal_status noalloc_scratch(void** out) {
+  int dev = 0;
+  WAVEAL_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return waveal::fail(WAVEAL_ERR_UNSUPPORTED, "device ordinal %d not supported", dev);
+  std::lock_guard<std::mutex> lock(g_scratch_mu);
+  if (!g_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess || !ptr)
+      return waveal::fail(WAVEAL_ERR_CUDA, "cudaGetSymbolAddress(static scratch) failed: %s", cudaGetErrorString(e));
+    g_scratch_addr[dev] = ptr;
+  }
+  *out = g_scratch_addr[dev];
+  return WAVEAL_OK;
+}
+}  // namespace
+
+extern "C" size_t waveal_noalloc_max_rows(void) { return WAVEAL_NOALLOC_SCRATCH_BYTES / 4 - 1; }
+
+extern "C" waveal_status waveal_bitmap_to_csr_noalloc(int32_t heads, int32_t n_q_blocks, int32_t n_kv_blocks,
+                                                      const uint64_t* mask_bits, int32_t* kv_row_ptr_out,
+                                                      int32_t* kv_block_indices_out, int64_t capacity,
+                                                      void* cuda_stream) {
+  if (heads <= 0 || n_q_blocks <= 0 || n_kv_blocks <= 0)
+    return waveal::fail(WAVEAL_ERR_INVALID_ARG, "heads, n_q_blocks and n_kv_blocks must be positive");
+  const long long rows = (long long)heads * n_q_blocks;
+  if ((unsigned long long)rows > (unsigned long long)waveal_noalloc_max_rows())
+    return waveal::fail(WAVEAL_ERR_UNSUPPORTED,
+                        "heads*n_q_blocks = %lld exceeds the %zu rows the built-in scratch holds; "
+                        "use waveal_bitmap_to_csr with a caller-owned workspace",
+                        rows, waveal_noalloc_max_rows());
+  void* scratch = nullptr;
+  waveal_status s = noalloc_scratch(&scratch);
+  if (s != WAVEAL_OK) return s;
+  // the per-row counts in the scratch are fully rewritten for the rows in use before they are
+  // read, so nothing of the previous call's contents has to be cleared
+  return waveal_bitmap_to_csr(heads, n_q_blocks, n_kv_blocks, mask_bits, kv_row_ptr_out, kv_block_indices_out,
+                              capacity, scratch, WAVEAL_NOALLOC_SCRATCH_BYTES, cuda_stream);
 }
