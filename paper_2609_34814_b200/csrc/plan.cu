@@ -134,7 +134,9 @@ __global__ void k_fill_indices(const u64* __restrict__ bits, long long n_rows, i
 
 // ------------------------------------------------------------------ block-wide helpers
 
-// Sum of N doubles per thread over the CTA, same result in every thread; fixed tree.
+// Sum of N doubles per thread over the CTA, same result in every thread; fixed tree
+// (lanes, then warps).  fp64 adds are scarce on this part, so the second level is one more
+// shuffle tree in warp 0, not a serial sum in every thread.
 template <int N>
 __device__ __forceinline__ void block_sum(double (&v)[N], double* scratch) {
   int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -148,12 +150,22 @@ __device__ __forceinline__ void block_sum(double (&v)[N], double* scratch) {
     for (int k = 0; k < N; ++k) scratch[warp * N + k] = v[k];
   }
   __syncthreads();
+  if (warp == 0) {
+    double t[N];
 #pragma unroll
-  for (int k = 0; k < N; ++k) {
-    double s = 0.0;
-    for (int w = 0; w < kPlanWarps; ++w) s += scratch[w * N + k];
-    v[k] = s;
+    for (int k = 0; k < N; ++k) {
+      t[k] = scratch[lane * N + k];           // kPlanWarps == 32: one partial per lane
+#pragma unroll
+      for (int o = 16; o; o >>= 1) t[k] += __shfl_xor_sync(0xffffffffu, t[k], o);
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int k = 0; k < N; ++k) scratch[kPlanWarps * N + k] = t[k];
+    }
   }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < N; ++k) v[k] = scratch[kPlanWarps * N + k];
   __syncthreads();
 }
 
@@ -207,44 +219,62 @@ __device__ __forceinline__ int popcount_range(const u64* __restrict__ words, int
 }
 
 // dst[r] = sum_{c : bit (r, c) set} src[c] - rowscale(r) * corr ; rowscale = cnt[r] or 1.
-// One warp takes four consecutive bit rows per step (four loads in flight per lane).
-__device__ __forceinline__ void gather_rows(const u64* __restrict__ bits, int n_rows, int wpr,
-                                            const double2* src, double2* dst,
-                                            const int* __restrict__ cnt, double2 corr) {
-  int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int r0 = warp * 4; r0 < n_rows; r0 += kPlanWarps * 4) {
-    double ax[4] = {0, 0, 0, 0}, ay[4] = {0, 0, 0, 0};
-    for (int w0 = 0; w0 < wpr; w0 += 32) {
-      int w = w0 + lane;
+// L lanes share one bit row (lane q of the group takes words q, q+L, ...), 32/L rows per warp
+// step; the partial sums meet in a fixed shuffle tree of width L.  Fewer lanes per row than a
+// whole warp keeps more rows in flight and wastes fewer of the scarce fp64 adds on the tree.
+template <int L>
+__device__ __forceinline__ void gather_rows_l(const u64* __restrict__ bits, int n_rows, int wpr,
+                                              const double2* src, double2* dst,
+                                              const int* __restrict__ cnt, double2 corr) {
+  constexpr int RPW = 32 / L;                       // rows per warp step
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp = lane / L, q = lane % L;
+  for (int r0 = warp * RPW; r0 < n_rows; r0 += kPlanWarps * RPW) {
+    const int r = r0 + grp;
+    const bool live = r < n_rows;
+    double ax = 0.0, ay = 0.0;
+    for (int w0 = 0; w0 < wpr; w0 += 4 * L) {
       u64 word[4];
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        word[k] = (r0 + k < n_rows && w < wpr) ? bits[(size_t)(r0 + k) * wpr + w] : 0ull;
+      for (int k = 0; k < 4; ++k) {
+        const int w = w0 + q + k * L;
+        word[k] = (live && w < wpr) ? bits[(size_t)r * wpr + w] : 0ull;
+      }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
+        const int base = (w0 + q + k * L) * 64;
         u64 x = word[k];
         while (x) {
-          int b = __ffsll((long long)x) - 1;
+          const int b = __ffsll((long long)x) - 1;
           x &= x - 1;
-          double2 v = src[w * 64 + b];
-          ax[k] += v.x;
-          ay[k] += v.y;
+          const double2 v = src[base + b];
+          ax += v.x;
+          ay += v.y;
         }
       }
     }
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-#pragma unroll
-      for (int o = 16; o; o >>= 1) {
-        ax[k] += __shfl_xor_sync(0xffffffffu, ax[k], o);
-        ay[k] += __shfl_xor_sync(0xffffffffu, ay[k], o);
-      }
-      if (lane == 0 && r0 + k < n_rows) {
-        double sc = cnt ? (double)cnt[r0 + k] : 1.0;
-        dst[r0 + k] = make_double2(ax[k] - sc * corr.x, ay[k] - sc * corr.y);
-      }
+    for (int o = L / 2; o; o >>= 1) {
+      ax += __shfl_xor_sync(0xffffffffu, ax, o);
+      ay += __shfl_xor_sync(0xffffffffu, ay, o);
+    }
+    if (live && q == 0) {
+      const double sc = cnt ? (double)cnt[r] : 1.0;
+      dst[r] = make_double2(ax - sc * corr.x, ay - sc * corr.y);
     }
   }
+}
+
+__device__ __forceinline__ void gather_rows(const u64* __restrict__ bits, int n_rows, int wpr,
+                                            const double2* src, double2* dst,
+                                            const int* __restrict__ cnt, double2 corr) {
+  // about three words per lane
+  if (wpr <= 3) gather_rows_l<1>(bits, n_rows, wpr, src, dst, cnt, corr);
+  else if (wpr <= 6) gather_rows_l<2>(bits, n_rows, wpr, src, dst, cnt, corr);
+  else if (wpr <= 12) gather_rows_l<4>(bits, n_rows, wpr, src, dst, cnt, corr);
+  else if (wpr <= 24) gather_rows_l<8>(bits, n_rows, wpr, src, dst, cnt, corr);
+  else if (wpr <= 48) gather_rows_l<16>(bits, n_rows, wpr, src, dst, cnt, corr);
+  else gather_rows_l<32>(bits, n_rows, wpr, src, dst, cnt, corr);
 }
 
 // Q factor of the thin QR of an m x 2 block: Gram-Schmidt with one re-orthogonalisation
@@ -343,8 +373,8 @@ struct PlanParams {
 
 __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_head(PlanParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
-  double* scratch = reinterpret_cast<double*>(smem);                 // 32*4 doubles
-  unsigned char* region = smem + 1024;
+  double* scratch = reinterpret_cast<double*>(smem);                 // (32 + 1) * 4 doubles
+  unsigned char* region = smem + 2048;
   const int h = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int m_b = p.m_b, n_b = p.n_b;
   const u64* M = p.M + (size_t)h * m_b * p.wq;
@@ -556,8 +586,8 @@ waveal_status plan_layout(const waveal_plan_desc* d, PlanLayout* L) {
   while (p2 < d->n_q_blocks) p2 <<= 1;
   L->n_pow2 = p2;
   size_t sort_bytes = (size_t)p2 * 12, state_bytes = (2 * m + n) * 16;
-  L->state_in_smem = 1024 + (state_bytes > sort_bytes ? state_bytes : sort_bytes) <= kSmemMax;
-  L->smem = 1024 + (L->state_in_smem ? (state_bytes > sort_bytes ? state_bytes : sort_bytes) : sort_bytes);
+  L->state_in_smem = 2048 + (state_bytes > sort_bytes ? state_bytes : sort_bytes) <= kSmemMax;
+  L->smem = 2048 + (L->state_in_smem ? (state_bytes > sort_bytes ? state_bytes : sort_bytes) : sort_bytes);
   size_t o = 0;
   L->off_bitmap = o; o = align_up(o + H * m * L->wq * 8, 256);
   L->off_mt = o;     o = align_up(o + H * n * L->wk * 8, 256);
