@@ -12,16 +12,13 @@
 //   warp 0      producer: takes tickets, publishes tasks, issues TMA loads of the Q tile and
 //               of the K/V tiles (128-byte-swizzled slabs) into a shared-memory ring
 //   warp 1      MMA issuer: S = Q K^T (operands in shared memory) and O += P V (P read from
-//               tensor memory) as tcgen05.mma with fp32 accumulators in tensor memory
-//   warps 2-5   softmax group 0: the even-numbered blocks of the row's list
-//   warps 6-9   softmax group 1: the odd-numbered blocks
-//               Each group owns one S/P buffer and one partial output in tensor memory and
-//               its own running (max, sum): while one group runs the softmax of block j the
-//               tensor cores work for the other (P_{j-1} V_{j-1}, then Q K_{j+1}^T).  A thread
-//               owns one row: it reads S, writes P (bf16) over the same columns, and rescales
-//               its partial O only when the max grew by more than 2^8.  The epilogue merges
-//               the two partial results exactly, normalises and stores O at the ORIGINAL row
-//               position (no inverse permutation pass).
+//               tensor memory) as tcgen05.mma with fp32 accumulators in tensor memory; three
+//               S buffers, so Q K_{j+1}^T and Q K_{j+2}^T are done while the softmax of S_j runs
+//   warps 2-9   softmax: thread (row, half) reads half a row of S from tensor memory, the two
+//               halves exchange their maxima through shared memory, then the thread writes P
+//               (bf16) over the columns S came from; the running max / sum stay in registers;
+//               O in tensor memory is rescaled only when the max grew by more than 2^8; the
+//               epilogue normalises and stores O at the ORIGINAL row (no inverse permutation)
 // Every wait on an mbarrier is bounded; when one runs out the CTA records
 // {WAVEAL_ERR_TIMEOUT, site} and all roles leave through the common teardown.
 #include <cuda.h>
@@ -34,6 +31,10 @@ namespace {
 constexpr int kThreads = 320;
 constexpr int kSoftmaxWarp0 = 2;
 constexpr long long kTimeoutCycles = 4000000000ll;   // ~2 s at boost clock
+#ifndef WAVEAL_POLY_EVERY
+#define WAVEAL_POLY_EVERY 0
+#endif
+constexpr int kPolyEvery = WAVEAL_POLY_EVERY;          // n > 0: 1 pair in n computes 2^x on the FMA pipe (0 = off: measured slower, the softmax is issue-bound)
 
 // ------------------------------------------------------------------ PTX wrappers
 
@@ -173,6 +174,15 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       ::WAVEAL_IN32(v, o), "r"(taddr)                                                            \
       : "memory")
 
+#define WAVEAL_TMEM_ST16(taddr, v, o)                                                            \
+  asm volatile(                                                                                  \
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "                                           \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"                  \
+      ::"r"(v[o+0]), "r"(v[o+1]), "r"(v[o+2]), "r"(v[o+3]), "r"(v[o+4]), "r"(v[o+5]), "r"(v[o+6]), "r"(v[o+7]), \
+        "r"(v[o+8]), "r"(v[o+9]), "r"(v[o+10]), "r"(v[o+11]), "r"(v[o+12]), "r"(v[o+13]), "r"(v[o+14]), "r"(v[o+15]), \
+        "r"(taddr)                                                                               \
+      : "memory")
+
 __device__ __forceinline__ float ex2(float x) {
 #ifdef WAVEAL_DBG_NOEXP
   return x * 0.001f + 0.5f;
@@ -182,6 +192,23 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 #endif
 }
+// 2^x on the FMA and integer pipes (for a share of the elements, to take load off the
+// transcendental pipe, which would otherwise be as busy as the tensor cores): round x to the
+// nearest integer n with the 1.5*2^23 trick, degree-3 polynomial for 2^(x-n) on [-0.5, 0.5]
+// (relative error 7.5e-5, far below the bf16 cut of P), n added to the exponent field.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fmaxf(x, -125.0f);
+  const float xi = x + 12582912.0f;
+  const float f = x - (xi - 12582912.0f);
+  float q = fmaf(0.05517137423157692f, f, 0.2426110953092575f);
+  q = fmaf(q, f, 0.6932610273361206f);
+  q = fmaf(q, f, 0.9999280571937561f);
+  return __int_as_float(__float_as_int(q) + (__float_as_int(xi) << 23));
+}
+// Register re-allocation between warpgroups (each scheduler hosts one warp of every
+// warpgroup): the producer/MMA warpgroup gives registers up, the softmax warpgroups take them.
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
@@ -198,6 +225,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 }
 
 // instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major
+// (A and B must have the same 16-bit format: an f16 A with a bf16 B is an illegal instruction)
 __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(m >> 4) << 24);
@@ -229,19 +257,25 @@ struct Geo {
   static constexpr int TILE_BYTES = SLABS * BK * 128;
   static constexpr int KV_SLAB_BYTES = BK * 128;
   static constexpr int NSTAGE_RAW = (200 * 1024 - Q_BYTES) / TILE_BYTES;
+#ifdef WAVEAL_DBG_NSTAGE
+  static constexpr int NSTAGE = WAVEAL_DBG_NSTAGE;
+#else
   static constexpr int NSTAGE = NSTAGE_RAW > 8 ? 8 : NSTAGE_RAW;
-  static constexpr int PC = BK / 2;                  // tensor-memory columns of a P tile (bf16 pairs)
-  static constexpr int CO = D / 2;                   // O columns per epilogue thread
+#endif
+  static constexpr int NSBUF = 3;                    // S/P buffers in tensor memory
+  static constexpr int CS = BK / 2;                  // S columns per softmax thread (half a row)
+  static constexpr int PC = BK / 4;                  // packed P columns per softmax thread
+  static constexpr int CO = D / 2;                   // O columns per softmax thread
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_KV = OFF_Q + Q_BYTES;
   static constexpr int OFF_BAR = OFF_KV + NSTAGE * TILE_BYTES;
-  static constexpr int N_BAR = 4 + 2 + 2 * NSTAGE + 2 + 2 + 3;
+  static constexpr int N_BAR = 4 + 2 + 2 * NSTAGE + 2 * NSBUF + 1 + 3;
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
-  static constexpr int OFF_EX = OFF_TASK + 2 * (int)sizeof(Task);
-  static constexpr int OFF_MISC = OFF_EX + 2 * 2 * 128 * 8;
+  static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
+  static constexpr int OFF_MISC = OFF_MX + 2 * 2 * 128 * 4;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for 1024-byte alignment
-  // tensor memory: two S/P buffers (even / odd K/V blocks) and the two partial outputs
-  static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL0 = 256, O_COL1 = 384, TMEM_COLS = 512;
+  // tensor memory: three S/P buffers and the output accumulator
+  static constexpr uint32_t S_STRIDE = 128, O_COL = 384, TMEM_COLS = 512;
 };
 
 #ifdef WAVEAL_TRACE
@@ -317,11 +351,11 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const uint32_t bar0 = sbase + G::OFF_BAR;
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   constexpr int B_TASK_FULL = 0, B_TASK_EMPTY = 2, B_Q_FULL = 4, B_Q_EMPTY = 5, B_KV_FULL = 6,
-                B_KV_EMPTY = 6 + G::NSTAGE, B_S_FULL = 6 + 2 * G::NSTAGE, B_P_FULL = B_S_FULL + 2,
-                B_O_FULL = B_P_FULL + 2, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1;
+                B_KV_EMPTY = 6 + G::NSTAGE, B_S_FULL = 6 + 2 * G::NSTAGE, B_P_FULL = B_S_FULL + G::NSBUF,
+                B_PV_DONE = B_P_FULL + G::NSBUF, B_O_FULL = B_PV_DONE + 1, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1;
   static_assert(B_FINAL + 1 <= G::N_BAR, "barrier count");
   Task* tasks = reinterpret_cast<Task*>(smem + G::OFF_TASK);
-  float2* ex = reinterpret_cast<float2*>(smem + G::OFF_EX);          // [task parity][group][128] (m, l)
+  float* mx = reinterpret_cast<float*>(smem + G::OFF_MX);            // [2][2][128] row-max / row-sum exchange
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + G::OFF_MISC);
   volatile int* abort_smem = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 4);
   Ctx ctx{bar0, abort_smem, p.ws, p.dev_status};
@@ -331,7 +365,10 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     mbar_init(BAR(B_Q_FULL), 1);
     mbar_init(BAR(B_Q_EMPTY), 1);
     for (int i = 0; i < G::NSTAGE; ++i) { mbar_init(BAR(B_KV_FULL + i), 1); mbar_init(BAR(B_KV_EMPTY + i), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_S_FULL + i), 1); mbar_init(BAR(B_P_FULL + i), 4); }
+    for (int i = 0; i < G::NSBUF; ++i) mbar_init(BAR(B_S_FULL + i), 1);
+    // one P barrier per S buffer: a warp may run up to two blocks ahead of the slowest one
+    for (int i = 0; i < G::NSBUF; ++i) mbar_init(BAR(B_P_FULL + i), 8);
+    mbar_init(BAR(B_PV_DONE), 1);
     mbar_init(BAR(B_O_FULL), 1);
     mbar_init(BAR(B_O_FREE), 8);
     mbar_init(BAR(B_FINAL), 1);
@@ -398,7 +435,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
       q_armed = true; q_armed_parity = q_it & 1;
       ++q_it;
-      // K/V tiles in the order the MMA warp consumes them: K_0, K_1, then V_j, K_{j+2} for each j
+      // K/V tiles in the order the MMA warp consumes them: K_0..K_2, then V_j, K_{j+3} for each j
       int chunk_base = -64, my_idx = 0;
       auto load_tile = [&](bool is_k, int j) -> bool {
         if (j < chunk_base || j >= chunk_base + 32) {
@@ -429,11 +466,10 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         ++kv_it;
         return true;
       };
-      ok = load_tile(true, 0);
-      if (ok && tk.n > 1) ok = load_tile(true, 1);
+      for (int j = 0; j < G::NSBUF && j < tk.n && ok; ++j) ok = load_tile(true, j);
       for (int j = 0; j < tk.n && ok; ++j) {
         ok = load_tile(false, j);
-        if (ok && j + 2 < tk.n) ok = load_tile(true, j + 2);
+        if (ok && j + G::NSBUF < tk.n) ok = load_tile(true, j + G::NSBUF);
       }
     }
     if (*abort_smem) {
@@ -457,8 +493,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     // compare-and-reset instead of modulo.
     constexpr uint32_t IDESC_QK = make_idesc(128, G::BK, false);
     constexpr uint32_t IDESC_PV = make_idesc(128, D, true);
-    uint32_t task_slot = 0, task_ph = 0, q_ph = 0, o_ph = 1, kv_st = 0, kv_ph = 0;
-    uint32_t p_ph0 = 0, p_ph1 = 0;
+    uint32_t task_slot = 0, task_ph = 0, q_ph = 0, o_ph = 1, kv_st = 0, kv_ph = 0, p_phase = 0;
     TRACE_DECL;
     const uint64_t qdesc0 = make_desc(sbase + G::OFF_Q, 16, 1024);
     const uint64_t kdesc0 = make_desc(sbase + G::OFF_KV, 16, 1024);
@@ -477,15 +512,15 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       ok = warp_wait(ctx, BAR(B_Q_FULL), q_ph, 11);
       if (!ok) break;
       q_ph ^= 1;
-      // S[g] = Q K_j^T (g = j & 1); overwrites the P tile that aliases S[g], which the
-      // preceding P V of the same parity (issued earlier by this warp) has consumed.
+      // S[sb] = Q K_j^T (sb = j mod 3); overwrites the P tile that aliases S[sb], which the
+      // P V three blocks earlier (issued before by this warp, executed in order) has consumed.
       // The caller has already waited for the K tile in stage kv_st.
-      auto issue_qk = [&](uint32_t g) {
+      auto issue_qk = [&](uint32_t sb) {
         TRACE(0, 4, (int)kv_st);
         {
           // descriptors differ from the per-kernel bases only in the 14-bit address field
           const uint64_t kd = kdesc0 + (uint64_t)(kv_st * (uint32_t)(G::TILE_BYTES >> 4));
-          const uint32_t d_s = tmem_base + g * 128u;
+          const uint32_t d_s = tmem_base + sb * G::S_STRIDE;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
 #ifndef WAVEAL_DBG_SKIP_QK
@@ -494,39 +529,36 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #endif
           }
           tc_commit(BAR(B_KV_EMPTY + kv_st));
-          tc_commit(BAR(B_S_FULL + g));
+          tc_commit(BAR(B_S_FULL + sb));
         }
         TRACE(0, 5, (int)kv_st);
         if (++kv_st == (uint32_t)G::NSTAGE) { kv_st = 0; kv_ph ^= 1; }
       };
-      ok = warp_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, 12);
-      if (!ok) break;
-      issue_qk(0);
-      if (n > 1) {
+      for (int j = 0; j < G::NSBUF && j < n && ok; ++j) {
         ok = warp_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, 12);
-        if (!ok) break;
-        issue_qk(1);
+        if (ok) issue_qk((uint32_t)j);
       }
-      if (n <= 2) tc_commit(BAR(B_Q_EMPTY));
-      // the partial outputs of the previous task have been read by the epilogue
+      if (!ok) break;
+      if (n <= G::NSBUF) tc_commit(BAR(B_Q_EMPTY));
+      // the output accumulator of the previous task has been read by the epilogue
       ok = warp_wait(ctx, BAR(B_O_FREE), o_ph, 16);
       if (!ok) break;
       o_ph ^= 1;
       // answers for the first P V of the task
-      uint32_t tok_p = mbar_test_wait(BAR(B_P_FULL + 0), p_ph0);
+      uint32_t tok_p = mbar_test_wait(BAR(B_P_FULL + 0), p_phase & 1u);
       uint32_t tok_v = mbar_test_wait(BAR(B_KV_FULL + kv_st), kv_ph);
+      uint32_t sb = 0;
       for (int j = 0; j < n && ok; ++j) {
-        const uint32_t g = (uint32_t)j & 1u;
-        // O[g] (+)= P_j V_j, P_j read from tensor memory
-        ok = finish_wait(ctx, BAR(B_P_FULL + g), g ? p_ph1 : p_ph0, tok_p, 14);
+        // O (+)= P_j V_j, P_j read from tensor memory
+        ok = finish_wait(ctx, BAR(B_P_FULL + sb), (p_phase >> sb) & 1u, tok_p, 14);
         if (!ok) break;
-        if (g) p_ph1 ^= 1; else p_ph0 ^= 1;
+        p_phase ^= 1u << sb;
         TRACE(0, 1, j);
         ok = finish_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, tok_v, 15);
         if (!ok) break;
         TRACE(0, 2, j);
-        const bool more_qk = j + 2 < n;
-        // the K tile of block j+2 sits in the stage after this V tile: ask now, use after the MMAs
+        const bool more_qk = j + G::NSBUF < n;
+        // the K tile of block j+3 sits in the stage after this V tile: ask now, use after the MMAs
         uint32_t k_st = kv_st + 1, k_ph = kv_ph;
         if (k_st == (uint32_t)G::NSTAGE) { k_st = 0; k_ph ^= 1; }
         uint32_t tok_k = more_qk ? mbar_test_wait(BAR(B_KV_FULL + k_st), k_ph) : 1u;
@@ -535,9 +567,9 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           // V tile as the N x K operand with N (head_dim) contiguous: 8 keys per 1024-byte
           // group along K (16 keys = 2048 bytes per MMA), next 64 columns of head_dim one slab further
           const uint64_t vd = vdesc0 + (uint64_t)(kv_st * (uint32_t)(G::TILE_BYTES >> 4));
-          const uint32_t pbase = tmem_base + g * 128u;
-          const uint32_t d_o = tmem_base + G::O_COL0 + g * 128u;
-          if (j >= 2) {
+          const uint32_t pbase = tmem_base + sb * G::S_STRIDE;
+          const uint32_t d_o = tmem_base + G::O_COL;
+          if (j > 0) {
 #pragma unroll
             for (int k = 0; k < G::BK / 16; ++k) {
 #ifndef WAVEAL_DBG_SKIP_PV
@@ -553,6 +585,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
           }
           tc_commit(BAR(B_KV_EMPTY + kv_st));
+          tc_commit(BAR(B_PV_DONE));
           if (j == n - 1) tc_commit(BAR(B_O_FULL));
         }
         TRACE(0, 3, j);
@@ -561,17 +594,19 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           ok = finish_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, tok_k, 12);
           if (!ok) break;
         }
-        // answers for the next P V (other group's P tile; its V tile follows the K tile just checked)
+        // answers for the next P V (its V tile follows the K tile just checked)
         if (j + 1 < n) {
           uint32_t v_st = kv_st, v_ph = kv_ph;
           if (more_qk) { if (++v_st == (uint32_t)G::NSTAGE) { v_st = 0; v_ph ^= 1; } }
-          tok_p = mbar_test_wait(BAR(B_P_FULL + (g ^ 1u)), g ? p_ph0 : p_ph1);
+          const uint32_t nsb = (sb + 1 == (uint32_t)G::NSBUF) ? 0u : sb + 1;
+          tok_p = mbar_test_wait(BAR(B_P_FULL + nsb), (p_phase >> nsb) & 1u);
           tok_v = mbar_test_wait(BAR(B_KV_FULL + v_st), v_ph);
         }
         if (more_qk) {
-          issue_qk(g);
-          if (j + 2 == n - 1) tc_commit(BAR(B_Q_EMPTY));
+          issue_qk(sb);
+          if (j + G::NSBUF == n - 1) tc_commit(BAR(B_Q_EMPTY));
         }
+        if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
     }
     // every MMA issued by this warp has completed before tensor memory is released
@@ -583,15 +618,16 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
   } else {
     // ============================================================== softmax / epilogue
-    // group 0 (warps 2-5) takes the even K/V blocks of a row's list, group 1 (warps 6-9) the
-    // odd ones; each keeps its own reference max, sum and partial output; the epilogue merges.
-    const int g = (warp - kSoftmaxWarp0) >> 2;
+    // All eight warps work on every block: thread (row, half) owns half a row of S, so two
+    // warps per scheduler interleave and hide each other's latencies; the two halves of a row
+    // exchange their maxima through shared memory (one 64-thread named barrier per block).
+    const int sw = warp - kSoftmaxWarp0;       // 0..7
     const int quad = warp & 3;                 // tensor-memory lane quadrant this warp may access
+    const int half = sw >> 2;                  // which half of the S / O columns
     const int r = quad * 32 + lane;            // row of the 128-row MMA tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t s_addr = tmem_base + lane_addr + (g ? G::S_COL1 : G::S_COL0);
-    const uint32_t o_own = tmem_base + lane_addr + (g ? G::O_COL1 : G::O_COL0);
-    uint32_t task_it = 0, s_it = 0, o_it = 0;
+    const uint32_t o_addr = tmem_base + lane_addr + G::O_COL + half * G::CO;
+    uint32_t task_it = 0, s_phase = 0, o_it = 0, pv_total = 0, blk_it = 0;
     TRACE_DECL;
     bool ok = true;
     while (ok) {
@@ -601,60 +637,64 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const Task tk = tasks[slot];
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + slot));
-      float2* exb = ex + (task_it & 1) * 256;
       ++task_it;
       if (tk.n < 0) break;
       const long long q_tok = (long long)tk.row * G::BQ + r;
       const bool row_live = r < G::BQ && q_tok < p.seq_q;
-      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + g * G::CO;
+      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + half * G::CO;
       if (tk.n == 0) {
         if (row_live) {
 #pragma unroll
           for (int c = 0; c < G::CO / 8; ++c) reinterpret_cast<uint4*>(o_ptr)[c] = make_uint4(0, 0, 0, 0);
-          if (p.lse && g == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
+          if (p.lse && half == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
         }
         continue;
       }
       float m_used = -INFINITY, l_run = 0.f;
-      for (int j = g; j < tk.n && ok; j += 2) {
-        ok = warp_wait(ctx, BAR(B_S_FULL + g), s_it & 1, 21);
+      uint32_t sb = 0;
+      for (int j = 0; j < tk.n && ok; ++j) {
+        ok = warp_wait(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
         if (!ok) break;
-        ++s_it;
-        if (quad == 2) TRACE(1 + g, 10 + g, j);
+        s_phase ^= 1u << sb;
+        if (sw == 2 || sw == 6) TRACE(1 + half, 10 + half, j);
         tc_fence_after();
-#ifdef WAVEAL_DBG_NOSOFTMAX
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_P_FULL + g));
-        continue;
-#endif
-        uint32_t sv[G::BK];
-#pragma unroll
-        for (int c = 0; c < G::BK; c += 32) WAVEAL_TMEM_LD32(s_addr + c, sv, c);
-#pragma unroll
-        for (int c = 0; c < G::BK; c += 32) WAVEAL_TMEM_WAIT_LD32(sv, c);
-        if (quad == 2) TRACE(1 + g, 12 + g, j);
+        const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE;
+        uint32_t sv[G::CS];
+        if constexpr (G::CS == 64) {
+          WAVEAL_TMEM_LD32(s_addr + half * 64, sv, 0);
+          WAVEAL_TMEM_LD32(s_addr + half * 64 + 32, sv, 32);
+          WAVEAL_TMEM_WAIT_LD32(sv, 0);
+          WAVEAL_TMEM_WAIT_LD32(sv, 32);
+        } else {
+          WAVEAL_TMEM_LD32(s_addr + half * 32, sv, 0);
+          WAVEAL_TMEM_WAIT_LD32(sv, 0);
+        }
+        if (sw == 2 || sw == 6) TRACE(1 + half, 12 + half, j);
         // scores of keys beyond seq_kv (ragged last block) do not exist
         if (j == tk.n - 1 && tk.tail_valid < G::BK) {
 #pragma unroll
-          for (int c = 0; c < G::BK; ++c)
-            if (c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
+          for (int c = 0; c < G::CS; ++c)
+            if (half * G::CS + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
         }
-        // row max with eight independent chains (a single chain of 128 dependent max ops
-        // would cost more than the exponentials)
+        // row max: eight independent chains, then the other half of the row through smem
         float mx8[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(sv[i]);
 #pragma unroll
-        for (int c = 8; c < G::BK; c += 8) {
+        for (int c = 8; c < G::CS; c += 8) {
 #pragma unroll
           for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(sv[c + i]));
         }
         const float mloc = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
                                  fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-        const float m_cand = fmaxf(m_used, mloc * p.sl2);
+        float* mxb = mx + (blk_it & 1) * 256;
+        ++blk_it;
+        mxb[half * 128 + r] = mloc;
+        named_bar_sync(1 + quad, 64);
+        const float m_cand = fmaxf(m_used, fmaxf(mloc, mxb[(half ^ 1) * 128 + r]) * p.sl2);
         // keep the stale reference max unless it is exceeded by more than 2^8 (exact: the
-        // final normalisation divides by a sum taken with the same reference)
+        // final normalisation divides by a sum taken with the same reference); both halves of a
+        // row see the same numbers and the two warps hold the same rows, so they decide alike
         const bool grow = __any_sync(0xffffffffu, m_cand > m_used + 8.0f);
         float alpha = 1.f;
         if (grow) {
@@ -670,85 +710,82 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         // the tensor core multiplies with, so numerator and denominator stay consistent.
         const float neg_m = ((m_used == -INFINITY) ? 0.f : -m_used) + 0.0028150156f;
 #pragma unroll
-        for (int c = 0; c < G::BK; c += 2) {
-          const uint32_t b0 = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c]), p.sl2, neg_m)));
-          const uint32_t b1 = __float_as_uint(ex2(fmaf(__uint_as_float(sv[c + 1]), p.sl2, neg_m)));
+        for (int c = 0; c < G::CS; c += 2) {
+          const float x0 = fmaf(__uint_as_float(sv[c]), p.sl2, neg_m);
+          const float x1 = fmaf(__uint_as_float(sv[c + 1]), p.sl2, neg_m);
+          // every kPolyEvery-th pair takes the polynomial path (a fixed pattern per column, so
+          // the result of a row does not depend on the execution order)
+          const bool poly = kPolyEvery > 0 && ((c >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == (kPolyEvery - 1);
+          const uint32_t b0 = __float_as_uint(poly ? ex2_fma(x0) : ex2(x0));
+          const uint32_t b1 = __float_as_uint(poly ? ex2_fma(x1) : ex2(x1));
           ls4[(c >> 1) & 3] += __uint_as_float(b0 & 0xFFFF0000u) + __uint_as_float(b1 & 0xFFFF0000u);
           pk[c / 2] = __byte_perm(b0, b1, 0x7632);
         }
-        const float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-        l_run += lsum;
-        if (quad == 2) TRACE(1 + g, 14 + g, j);
-        // P_j (bf16 pairs) over the first half of the columns of S[g]
+        l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+        if (sw == 2 || sw == 6) TRACE(1 + half, 14 + half, j);
+        // rare: the reference grew, so the accumulated O is rescaled; P_{j-1} V_{j-1} (the last MMA
+        // that touches O) must be complete - the barrier has seen exactly pv_total + j - 1 or
+        // pv_total + j phases by now, so a parity wait is unambiguous
+        if (grow && j > 0) {
+          ok = warp_wait(ctx, BAR(B_PV_DONE), (pv_total + (uint32_t)j - 1u) & 1u, 22);
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < G::PC; c += 32) WAVEAL_TMEM_ST32(s_addr + c, pk, c);
-        // S_FULL of block j implies that P V of block j-2 is complete: O[g] may be rescaled
-        if (grow && j >= 2) {
-#pragma unroll
-          for (int c0 = 0; c0 < D; c0 += 32) {
+          for (int c0 = 0; c0 < G::CO; c0 += 32) {
             uint32_t ov[32];
-            WAVEAL_TMEM_LD32(o_own + c0, ov, 0);
+            WAVEAL_TMEM_LD32(o_addr + c0, ov, 0);
             WAVEAL_TMEM_WAIT_LD32(ov, 0);
 #pragma unroll
             for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-            WAVEAL_TMEM_ST32(o_own + c0, ov, 0);
+            WAVEAL_TMEM_ST32(o_addr + c0, ov, 0);
           }
         }
+        // P_j (bf16 pairs) over the first half of the columns of S[sb]
+        if constexpr (G::PC == 32) { WAVEAL_TMEM_ST32(s_addr + half * 32, pk, 0); }
+        else { WAVEAL_TMEM_ST16(s_addr + half * 16, pk, 0); }
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_P_FULL + g));
-        if (quad == 2) TRACE(1 + g, 16 + g, j);
+        if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb));
+        if (sw == 2 || sw == 6) TRACE(1 + half, 16 + half, j);
+        if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
       if (!ok) break;
-      // ---- epilogue: merge the two partial results, normalise, store at the original rows
+      pv_total += (uint32_t)tk.n;
+      // ---- epilogue: O / l at the original row position
       ok = warp_wait(ctx, BAR(B_O_FULL), o_it & 1, 23);
       if (!ok) break;
       ++o_it;
       tc_fence_after();
-      if (quad == 2) TRACE(1 + g, 18 + g, tk.n);
-      exb[g * 128 + r] = make_float2(m_used, l_run);
+      if (sw == 2 || sw == 6) TRACE(1 + half, 18 + half, tk.n);
+      float* lx = mx + (blk_it & 1) * 256;      // the buffer the last block did not use
+      ++blk_it;
+      lx[half * 128 + r] = l_run;
       named_bar_sync(1 + quad, 64);
-      const float2 oth = exb[(g ^ 1) * 128 + r];
-      const float m_all = fmaxf(m_used, oth.x);
-      const float a_self = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_all);
-      const float a_oth = (oth.x == -INFINITY) ? 0.f : ex2(oth.x - m_all);
-      const float l_tot = a_self * l_run + a_oth * oth.y;
+      const float l_tot = l_run + lx[(half ^ 1) * 128 + r];
       const float inv_l = 1.0f / l_tot;
-      const float w_e = (g == 0 ? a_self : a_oth) * inv_l, w_o = (g == 0 ? a_oth : a_self) * inv_l;
-      uint32_t oe[G::CO], oo[G::CO];
-      const uint32_t col0 = tmem_base + lane_addr + g * G::CO;
+      uint32_t ov[G::CO];
 #pragma unroll
-      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(col0 + G::O_COL0 + c, oe, c);
-      if (tk.n >= 2) {
+      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(o_addr + c, ov, c);
 #pragma unroll
-        for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(col0 + G::O_COL1 + c, oo, c);
-#pragma unroll
-        for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(oo, c);
-      } else {
-#pragma unroll
-        for (int c = 0; c < G::CO; ++c) oo[c] = 0u;
-      }
-#pragma unroll
-      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(oe, c);
+      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(ov, c);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_O_FREE));
-      if (quad == 2) TRACE(1 + g, 30 + g, tk.n);
+      if (sw == 2 || sw == 6) TRACE(1 + half, 30 + half, tk.n);
       if (row_live) {
 #pragma unroll
         for (int c = 0; c < G::CO; c += 8) {
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            float x0 = __uint_as_float(oe[c + 2 * e]) * w_e + __uint_as_float(oo[c + 2 * e]) * w_o;
-            float x1 = __uint_as_float(oe[c + 2 * e + 1]) * w_e + __uint_as_float(oo[c + 2 * e + 1]) * w_o;
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(x0, x1);
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(ov[c + 2 * e]) * inv_l,
+                                                      __uint_as_float(ov[c + 2 * e + 1]) * inv_l);
             w[e] = *reinterpret_cast<uint32_t*>(&b2);
           }
           *reinterpret_cast<uint4*>(o_ptr + c) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (p.lse && g == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_all + log2f(l_tot)) * 0.6931471805599453f;
+        if (p.lse && half == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_used + log2f(l_tot)) * 0.6931471805599453f;
       }
     }
   }
