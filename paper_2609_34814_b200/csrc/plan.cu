@@ -240,16 +240,21 @@ __device__ __forceinline__ void gather_rows_l(const u64* __restrict__ bits, int 
         const int w = w0 + q + k * L;
         word[k] = (live && w < wpr) ? bits[(size_t)r * wpr + w] : 0ull;
       }
+      // walk the set bits of each word as two 32-bit halves (64-bit bit tricks cost twice
+      // the integer instructions, and this loop is bound by them)
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const int base = (w0 + q + k * L) * 64;
-        u64 x = word[k];
-        while (x) {
-          const int b = __ffsll((long long)x) - 1;
-          x &= x - 1;
-          const double2 v = src[base + b];
-          ax += v.x;
-          ay += v.y;
+        const double2* sp = src + (w0 + q + k * L) * 64;
+#pragma unroll
+        for (int hw = 0; hw < 2; ++hw) {
+          unsigned x = hw ? (unsigned)(word[k] >> 32) : (unsigned)word[k];
+          while (x) {
+            const int b = __ffs((int)x) - 1;
+            x &= x - 1;
+            const double2 v = sp[hw * 32 + b];
+            ax += v.x;
+            ay += v.y;
+          }
         }
       }
     }
