@@ -191,7 +191,9 @@ def run_waveal(args, cfg):
     ptr = torch.from_numpy(ptr_np).to(dev)
     idx = torch.from_numpy(idx_np).to(dev)
     W = wb.default_wave_size()
-    pdesc = wb.plan_desc_default(heads=H, n_q_blocks=nb, n_kv_blocks=nb, wave_size=W, mode=wb.FORCE_REORDER,
+    step_mode = {"reorder": wb.FORCE_REORDER, "natural": wb.FORCE_NATURAL, "auto": wb.AUTO,
+                 "stage1": wb.STAGE1_ONLY, "stage2": wb.STAGE2_ONLY}[args.plan_mode]
+    pdesc = wb.plan_desc_default(heads=H, n_q_blocks=nb, n_kv_blocks=nb, wave_size=W, mode=step_mode,
                                  seed=cfg.plan_seed, kv_bytes_per_head=2 * Sp * D * 2)
     pws = torch.empty((wb.plan_workspace_bytes(pdesc) + 256,), dtype=torch.uint8, device=dev)
     aws = torch.empty((256,), dtype=torch.uint8, device=dev)
@@ -200,7 +202,7 @@ def run_waveal(args, cfg):
     stream = torch.cuda.current_stream()
     launches = {"n": 0}
 
-    def step(mode=wb.FORCE_REORDER, count=False):
+    def step(mode=step_mode, count=False):
         pdesc.mode = mode
         plan = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream)
         if count:
@@ -219,7 +221,7 @@ def run_waveal(args, cfg):
     torch.cuda.synchronize()
     # ---- timed region: K steps, events on the launching stream; the attention kernel of each
     #      step is bracketed by its own events for the roofline figure
-    pdesc.mode = wb.FORCE_REORDER
+    pdesc.mode = step_mode
     attn_ev = []
     wd.barrier()
     torch.cuda.synchronize()
@@ -257,7 +259,8 @@ def run_waveal(args, cfg):
             ts.append(a.elapsed_time(b))
         return statistics.median(ts)
 
-    reo = plan.row_order
+    pdesc.mode = wb.FORCE_REORDER
+    reo = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream).row_order
     t_reo = timed(lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=reo, workspace=aws, dev_status=status, stream=stream))
     t_nat = timed(lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=None, workspace=aws, dev_status=status, stream=stream))
     t_plan = timed(lambda: wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream))
@@ -266,7 +269,7 @@ def run_waveal(args, cfg):
     torch.cuda.synchronize()
     skipped = int((auto.skip_flags & 1).sum().item())
     t_plan_auto = timed(lambda: wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream))
-    pdesc.mode = wb.FORCE_REORDER
+    pdesc.mode = step_mode
 
     # ---- end to end through the public API with host buffers: H2D of Q, K, V and the mask,
     #      index lists built on the device, plan, attention, D2H of O - all inside the timed region
@@ -310,7 +313,7 @@ def run_waveal(args, cfg):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "heads": H, "head_dim": D, "seq": S, "block": B, "block_pairs": pairs,
-                   "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": "FORCE_REORDER",
+                   "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode,
                    "step": "plan + attention", "l2": "inputs (Q,K,V,O %.1f GB) larger than L2, no flush" %
                    (4 * H * Sp * D * 2 / 1e9), "batch_elements": world},
         "roofline": {"bound": "tensor", "kernel": "k_bsattn_fwd", "achieved": achieved, "peak": pk["bf16"],
@@ -341,6 +344,8 @@ def main():
     ap.add_argument("--impl", default="waveal", choices=["waveal", "reference"])
     ap.add_argument("--config", default="wan720p")
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling / parity cases)")
+    ap.add_argument("--plan-mode", default="reorder", choices=["reorder", "natural", "auto", "stage1", "stage2"],
+                    help="which stages the plan of the timed step runs (Section 6.5 ablation); the headline is 'reorder'")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -660,7 +660,7 @@ extern "C" void waveal_plan_desc_default(waveal_plan_desc* d) {
   *d = waveal_plan_desc{};
   d->svd_iters = 10;
   d->mode = WAVEAL_AUTO;
-  d->l2_fit_num = 1; d->l2_fit_den = 2;
+  d->l2_fit_num = 1; d->l2_fit_den = 4;
   d->min_density_ppm = 10000;
   d->local_num = 1; d->local_den = 2;
   d->min_nnz = 0;

@@ -237,7 +237,7 @@ def test_guard_cases():
     # short sequence: the head's K+V fit the cache budget
     f = wo.guard_flags(mk, 8, {**g, "kv_bytes_per_head": 10, "l2_bytes": 100})
     assert f & wo.FLAG_SHORT_SEQ
-    f = wo.guard_flags(mk, 8, {**g, "kv_bytes_per_head": 51, "l2_bytes": 100})
+    f = wo.guard_flags(mk, 8, {**g, "kv_bytes_per_head": 26, "l2_bytes": 100})
     assert not f & wo.FLAG_SHORT_SEQ
     # too sparse
     sparse = np.eye(200, dtype=bool)
