@@ -270,6 +270,11 @@ def run_waveal(args, cfg):
     skipped = int((auto.skip_flags & 1).sum().item())
     t_plan_auto = timed(lambda: wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream))
     pdesc.mode = step_mode
+    # the two extra passes of the paper's own deployment (gather Q into the order, scatter O back),
+    # which the index-list kernel does not need: pure HBM copies, reported for context
+    t_gather = timed(lambda: wb.gather_rows(q, o, reo, B, stream=stream))
+    t_scatter = timed(lambda: wb.scatter_rows(q, o, reo, B, stream=stream))
+    copy_bytes = 2.0 * H * Sp * D * 2
 
     # ---- end to end through the public API with host buffers: H2D of Q, K, V and the mask,
     #      index lists built on the device, plan, attention, D2H of O - all inside the timed region
@@ -303,10 +308,10 @@ def run_waveal(args, cfg):
         e2e = {"value": world * flops / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": o_h.numel() * 2}
 
+    pk = peaks()
     if rank != 0:
         wd.shutdown()
         return
-    pk = peaks()
     achieved = flops / (attn_ms * 1e-3) / 1e12
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -323,7 +328,9 @@ def run_waveal(args, cfg):
         "kernel": {"attn_ms_reordered": t_reo, "attn_ms_natural": t_nat, "speedup_vs_natural": t_nat / t_reo,
                    "tflops_reordered": flops / t_reo / 1e9, "tflops_natural": flops / t_nat / 1e9,
                    "plan_ms": t_plan, "plan_ms_auto": t_plan_auto, "auto_skipped_heads": skipped,
-                   "plan_share_of_step": t_plan / (t_plan + t_reo)},
+                   "plan_share_of_step": t_plan / (t_plan + t_reo),
+                   "paper_gather_q_ms": t_gather, "paper_scatter_o_ms": t_scatter,
+                   "gather_gbs": copy_bytes / t_gather / 1e6, "gather_frac_of_hbm_peak": copy_bytes / t_gather / 1e6 / pk["hbm"]},
         "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
     }
     if world == 1 and not args.no_cpu:

@@ -185,6 +185,22 @@ waveal_status waveal_bsattn_fwd(const waveal_attn_desc* desc /*host*/, const voi
                                 float scale, void* ws /*dev*/, size_t ws_bytes, int32_t* dev_status /*dev or NULL*/,
                                 void* cuda_stream);
 
+/* The two reorder operators of the paper's deployment (Section 5), for driving a backend
+ * that cannot follow an index list: gather moves block row_order[h][p] of `src` to position p
+ * of `dst` (query blocks, or mask rows with block = 1 and row_bytes = bytes of a bitmap row
+ * padded to 16); scatter is the inverse (output block at position p goes back to block
+ * row_order[h][p]).  Tensors are [heads][n_blocks*block rows][row_bytes] with byte strides
+ * {head, row} (multiples of 16); src and dst must not overlap.  Pure copies: out-of-range
+ * entries of row_order move nothing.  waveal_bsattn_fwd itself needs neither pass. */
+waveal_status waveal_gather_rows(int32_t heads, int32_t n_blocks, int32_t block, int32_t row_bytes,
+                                 const void* src /*dev*/, const int64_t* src_stride_bytes /*host [2]*/,
+                                 void* dst /*dev*/, const int64_t* dst_stride_bytes /*host [2]*/,
+                                 const int32_t* row_order /*dev [heads][n_blocks]*/, void* cuda_stream);
+waveal_status waveal_scatter_rows(int32_t heads, int32_t n_blocks, int32_t block, int32_t row_bytes,
+                                  const void* src /*dev*/, const int64_t* src_stride_bytes /*host [2]*/,
+                                  void* dst /*dev*/, const int64_t* dst_stride_bytes /*host [2]*/,
+                                  const int32_t* row_order /*dev [heads][n_blocks]*/, void* cuda_stream);
+
 /* Number of query-block tasks the attention kernel keeps in flight on the current device
  * (SM count x CTAs per SM): the W to plan with (Section 6.1).  Returns <= 0 on failure. */
 int32_t waveal_default_wave_size(void);

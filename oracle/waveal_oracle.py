@@ -300,6 +300,21 @@ def plan_head(mask: np.ndarray, wave: int, iters: int, seed: int, head: int,
     return res
 
 
+def gather_blocks(x: np.ndarray, order: np.ndarray, block: int) -> np.ndarray:
+    """Reorder operator of Section 5: block p of the result is block order[p] of x
+    (x: [n_blocks*block, ...])."""
+    n = len(order)
+    return x.reshape(n, block, *x.shape[1:])[order].reshape(x.shape)
+
+
+def scatter_blocks(x: np.ndarray, order: np.ndarray, block: int) -> np.ndarray:
+    """Inverse operator of Section 5: block order[p] of the result is block p of x."""
+    n = len(order)
+    out = np.empty_like(x).reshape(n, block, *x.shape[1:])
+    out[order] = x.reshape(n, block, *x.shape[1:])
+    return out.reshape(x.shape)
+
+
 # ----------------------------------------------------------------------------- wave model
 
 

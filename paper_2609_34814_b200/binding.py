@@ -20,7 +20,7 @@ FLAG_SKIPPED, FLAG_SHORT_SEQ, FLAG_TOO_SPARSE, FLAG_ALREADY_LOCAL = 1, 2, 4, 8
 
 EXPORTS = ["waveal_plan_desc_default", "waveal_plan_workspace_bytes", "waveal_plan_bitmap", "waveal_plan_csr",
            "waveal_bitmap_to_csr", "waveal_bitmap_to_csr_noalloc", "waveal_noalloc_max_rows",
-           "waveal_bsattn_workspace_bytes", "waveal_bsattn_fwd",
+           "waveal_gather_rows", "waveal_scatter_rows", "waveal_bsattn_workspace_bytes", "waveal_bsattn_fwd",
            "waveal_default_wave_size", "waveal_last_launch_count", "waveal_status_string", "waveal_last_error"]
 
 
@@ -73,11 +73,14 @@ def load() -> ctypes.CDLL:
         lib.waveal_bitmap_to_csr_noalloc.argtypes = [I32, I32, I32, P, P, P, I64, P]
         lib.waveal_bitmap_to_csr_noalloc.restype = ctypes.c_int
         lib.waveal_noalloc_max_rows.restype = ctypes.c_size_t
+        for name in ("waveal_gather_rows", "waveal_scatter_rows"):
+            getattr(lib, name).argtypes = [I32, I32, I32, I32, P, ctypes.POINTER(I64), P, ctypes.POINTER(I64), P, P]
+            getattr(lib, name).restype = ctypes.c_int
         lib.waveal_bsattn_workspace_bytes.argtypes = [ctypes.POINTER(AttnDesc), ctypes.POINTER(ctypes.c_size_t)]
         lib.waveal_bsattn_fwd.argtypes = [ctypes.POINTER(AttnDesc), P, P, P, P, P, P, P, P, ctypes.c_float, P,
                                           ctypes.c_size_t, P, P]
         for name in ["waveal_plan_workspace_bytes", "waveal_plan_bitmap", "waveal_plan_csr", "waveal_bitmap_to_csr",
-                     "waveal_bsattn_workspace_bytes", "waveal_bsattn_fwd", "waveal_default_wave_size",
+                     "waveal_gather_rows", "waveal_scatter_rows", "waveal_bsattn_workspace_bytes", "waveal_bsattn_fwd", "waveal_default_wave_size",
                      "waveal_last_launch_count"]:
             getattr(lib, name).restype = ctypes.c_int
         lib.waveal_status_string.argtypes = [ctypes.c_int]
@@ -219,6 +222,27 @@ def bitmap_to_csr_noalloc(mask_bits, n_kv_blocks: int, kv_row_ptr, kv_block_indi
     cap = 0 if kv_block_indices is None else kv_block_indices.numel()
     _check(load().waveal_bitmap_to_csr_noalloc(H, M, n_kv_blocks, _ptr(mask_bits), _ptr(kv_row_ptr),
                                                _ptr(kv_block_indices), cap, _stream(stream)))
+
+
+def _move_rows(fn_name: str, src, dst, row_order, block: int, stream=None):
+    """src, dst: [heads, n_blocks*block, row elements] tensors (last dim contiguous)."""
+    H, rows, _ = src.shape
+    assert src.stride(2) == 1 and dst.stride(2) == 1 and dst.shape == src.shape
+    es = src.element_size()
+    ss = (ctypes.c_int64 * 2)(src.stride(0) * es, src.stride(1) * es)
+    ds = (ctypes.c_int64 * 2)(dst.stride(0) * es, dst.stride(1) * es)
+    _check(getattr(load(), fn_name)(H, rows // block, block, src.shape[2] * es, _ptr(src), ss, _ptr(dst), ds,
+                                    _ptr(row_order), _stream(stream)))
+
+
+def gather_rows(src, dst, row_order, block: int, stream=None):
+    """waveal_gather_rows: dst block p <- src block row_order[h][p]."""
+    _move_rows("waveal_gather_rows", src, dst, row_order, block, stream)
+
+
+def scatter_rows(src, dst, row_order, block: int, stream=None):
+    """waveal_scatter_rows: dst block row_order[h][p] <- src block p."""
+    _move_rows("waveal_scatter_rows", src, dst, row_order, block, stream)
 
 
 def attn_desc(q, k, v, o, seq_q: int, seq_kv: int, block: int, interleaved: bool = False) -> AttnDesc:

@@ -274,3 +274,13 @@ def test_lru_model_orders_the_ablation_as_the_paper_does():
     full = wo.lru_wave_model(mk, np.arange(mk.shape[0]), W, mk.shape[1])
     assert full["accesses"] == int(mk.sum())
     assert full["accesses"] - full["hits"] == int(mk.any(axis=0).sum())
+
+
+def test_gather_scatter_blocks_are_inverse_and_match_loops():
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((6 * 4, 3))
+    order = rng.permutation(6)
+    g = wo.gather_blocks(x, order, 4)
+    for p in range(6):
+        assert np.array_equal(g[p * 4:(p + 1) * 4], x[order[p] * 4:(order[p] + 1) * 4])
+    assert np.array_equal(wo.scatter_blocks(g, order, 4), x)
