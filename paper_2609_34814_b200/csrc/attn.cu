@@ -8,17 +8,23 @@
 // SM, take tickets from a global counter, so a freed SM starts the next row of the list at
 // once - the streaming "wave" behaviour of Section 2.3 that the schedule is built for.
 //
-// Structure of one CTA (320 threads):
+// Structure of one CTA (352 threads):
 //   warp 0      producer: takes tickets, publishes tasks, issues TMA loads of the Q tile and
-//               of the K/V tiles (128-byte-swizzled slabs) into a shared-memory ring
-//   warp 1      MMA issuer: S = Q K^T (operands in shared memory) and O += P V (P read from
-//               tensor memory) as tcgen05.mma with fp32 accumulators in tensor memory; three
-//               S buffers, so Q K_{j+1}^T and Q K_{j+2}^T are done while the softmax of S_j runs
-//   warps 2-9   softmax: thread (row, half) reads half a row of S from tensor memory, the two
-//               halves exchange their maxima through shared memory, then the thread writes P
-//               (bf16) over the columns S came from; the running max / sum stay in registers;
+//               of the K and V tiles (128-byte-swizzled slabs) into two shared-memory rings
+//   warp 10     MMA issuer 1: S_j = Q K_j^T (operands in shared memory) into one of three S
+//               buffers in tensor memory, up to three blocks ahead of the softmax
+//   warp 1      MMA issuer 2: O += P_j V_j (P read from tensor memory, where it lies over the
+//               columns S_j came from), fp32 accumulator in tensor memory.  Two issuing warps:
+//               the waits and ring arithmetic of one run while the other's MMAs execute
+//   warps 2-9   softmax, two teams of four warps that take the KV blocks of a task in turn:
+//               a thread owns one row of S for its team's blocks (row max, then exponentials
+//               and P in a second read of S); on every scheduler one warp of each team is
+//               resident, half a block apart, so one team's waits and loads hide behind the
+//               other's arithmetic.  The teams hand each other the running reference max of
+//               every row through shared memory; each keeps the row sum of its own blocks;
 //               O in tensor memory is rescaled only when the max grew by more than 2^8; the
-//               epilogue normalises and stores O at the ORIGINAL row (no inverse permutation)
+//               epilogue adds the two sums, normalises and stores O at the ORIGINAL row (no
+//               inverse permutation)
 // Every wait on an mbarrier is bounded; when one runs out the CTA records
 // {WAVEAL_ERR_TIMEOUT, site} and all roles leave through the common teardown.
 #include <cuda.h>
@@ -28,13 +34,13 @@
 
 namespace {
 
-constexpr int kThreads = 320;
-constexpr int kSoftmaxWarp0 = 2;
+constexpr int kThreads = 352;
+constexpr int kProducerWarp = 0, kPvWarp = 1, kSoftmaxWarp0 = 2, kQkWarp = 10;
 constexpr long long kTimeoutCycles = 4000000000ll;   // ~2 s at boost clock
 #ifndef WAVEAL_POLY_EVERY
-#define WAVEAL_POLY_EVERY 0
+#define WAVEAL_POLY_EVERY 2
 #endif
-constexpr int kPolyEvery = WAVEAL_POLY_EVERY;          // n > 0: 1 pair in n computes 2^x on the FMA pipe (0 = off: measured slower, the softmax is issue-bound)
+constexpr int kPolyEvery = WAVEAL_POLY_EVERY;          // n > 0: 1 pair of elements in n takes 2^x from the FMA pipe (0 = all from the transcendental unit)
 
 // ------------------------------------------------------------------ PTX wrappers
 
@@ -138,6 +144,37 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       : "memory");
 }
 
+// two fp32 operations per instruction (register pairs)
+__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2,%3};\n\tmov.b64 rb, {%4,%5};\n\tmov.b64 rc, {%6,%7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0,%1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void fadd2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2,%3};\n\tmov.b64 rb, {%4,%5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0,%1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
+// 2^x for two values on the FMA and integer pipes (for a share of the elements, to take load
+// off the transcendental unit: at 16 results per clock and SM it is as busy as the tensor
+// cores): x is rounded to the nearest integer n with the 1.5*2^23 trick, a degree-3 polynomial
+// gives 2^(x-n) on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16 cut of P), and n is
+// added to the exponent field.  Multiply-adds work on register pairs.
+__device__ __forceinline__ void ex2_fma2(float& e0, float& e1, float x0, float x1) {
+  x0 = fmaxf(x0, -125.0f);
+  x1 = fmaxf(x1, -125.0f);
+  float xi0, xi1, n0, n1, f0, f1, q0, q1;
+  fadd2(xi0, xi1, x0, x1, 12582912.0f, 12582912.0f);
+  fadd2(n0, n1, xi0, xi1, -12582912.0f, -12582912.0f);
+  ffma2(f0, f1, n0, n1, -1.0f, -1.0f, x0, x1);
+  ffma2(q0, q1, f0, f1, 0.05517137423157692f, 0.05517137423157692f, 0.2426110953092575f, 0.2426110953092575f);
+  ffma2(q0, q1, q0, q1, f0, f1, 0.6932610273361206f, 0.6932610273361206f);
+  ffma2(q0, q1, q0, q1, f0, f1, 0.9999280571937561f, 0.9999280571937561f);
+  e0 = __int_as_float(__float_as_int(q0) + (__float_as_int(xi0) << 23));
+  e1 = __int_as_float(__float_as_int(q1) + (__float_as_int(xi1) << 23));
+}
+
 #define WAVEAL_R32(v, o) \
   "=r"(v[o+0]), "=r"(v[o+1]), "=r"(v[o+2]), "=r"(v[o+3]), "=r"(v[o+4]), "=r"(v[o+5]), "=r"(v[o+6]), "=r"(v[o+7]), \
   "=r"(v[o+8]), "=r"(v[o+9]), "=r"(v[o+10]), "=r"(v[o+11]), "=r"(v[o+12]), "=r"(v[o+13]), "=r"(v[o+14]), "=r"(v[o+15]), \
@@ -192,23 +229,6 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 #endif
 }
-// 2^x on the FMA and integer pipes (for a share of the elements, to take load off the
-// transcendental pipe, which would otherwise be as busy as the tensor cores): round x to the
-// nearest integer n with the 1.5*2^23 trick, degree-3 polynomial for 2^(x-n) on [-0.5, 0.5]
-// (relative error 7.5e-5, far below the bf16 cut of P), n added to the exponent field.
-__device__ __forceinline__ float ex2_fma(float x) {
-  x = fmaxf(x, -125.0f);
-  const float xi = x + 12582912.0f;
-  const float f = x - (xi - 12582912.0f);
-  float q = fmaf(0.05517137423157692f, f, 0.2426110953092575f);
-  q = fmaf(q, f, 0.6932610273361206f);
-  q = fmaf(q, f, 0.9999280571937561f);
-  return __int_as_float(__float_as_int(q) + (__float_as_int(xi) << 23));
-}
-// Register re-allocation between warpgroups (each scheduler hosts one warp of every
-// warpgroup): the producer/MMA warpgroup gives registers up, the softmax warpgroups take them.
-template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
@@ -262,19 +282,22 @@ struct Geo {
 #else
   static constexpr int NSTAGE = NSTAGE_RAW > 8 ? 8 : NSTAGE_RAW;
 #endif
+  static constexpr int NKS = (NSTAGE + 1) / 2;       // K tile ring
+  static constexpr int NVS = NSTAGE / 2;             // V tile ring
   static constexpr int NSBUF = 3;                    // S/P buffers in tensor memory
-  static constexpr int CS = BK / 2;                  // S columns per softmax thread (half a row)
-  static constexpr int PC = BK / 4;                  // packed P columns per softmax thread
-  static constexpr int CO = D / 2;                   // O columns per softmax thread
+  static constexpr int CH = BK < 64 ? BK : 64;       // S columns a softmax thread holds at a time
+  static constexpr int NCH = BK / CH;                // such chunks per row
+  static constexpr int CO = D / 2;                   // O columns per epilogue thread
   static constexpr int OFF_Q = 0;
-  static constexpr int OFF_KV = OFF_Q + Q_BYTES;
-  static constexpr int OFF_BAR = OFF_KV + NSTAGE * TILE_BYTES;
-  static constexpr int N_BAR = 4 + 2 + 2 * NSTAGE + 2 * NSBUF + 1 + 3;
+  static constexpr int OFF_K = OFF_Q + Q_BYTES;
+  static constexpr int OFF_V = OFF_K + NKS * TILE_BYTES;
+  static constexpr int OFF_BAR = OFF_V + NVS * TILE_BYTES;
+  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 3 * NSBUF + 2 + 1 + 8;
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
   static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
-  static constexpr int OFF_MISC = OFF_MX + 2 * 2 * 128 * 4;
+  static constexpr int OFF_MISC = OFF_MX + 2 * 128 * 4 + 2 * 2 * 128 * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for 1024-byte alignment
-  // tensor memory: three S/P buffers and the output accumulator
+  // tensor memory: three S/P buffers of 128 columns, then the output accumulator
   static constexpr uint32_t S_STRIDE = 128, O_COL = 384, TMEM_COLS = 512;
 };
 
@@ -329,12 +352,22 @@ __device__ __forceinline__ bool warp_wait(const Ctx& c, uint32_t bar, uint32_t p
   return __all_sync(0xffffffffu, mbar_wait(c, bar, parity, site));
 }
 
-// Second half of a split wait: `tok` is the answer of a non-blocking probe issued earlier (before the
-// preceding group of MMAs, so that its latency hides behind their issue: the tensor pipe's
-// queue is short, and any pause of the issuing warp between two MMAs starves it).
-__device__ __forceinline__ bool finish_wait(const Ctx& c, uint32_t bar, uint32_t parity, uint32_t tok, int site) {
-  if (__all_sync(0xffffffffu, tok)) return true;
-  return warp_wait(c, bar, parity, site);
+// Latency-critical variant: polls with the non-suspending probe.  A suspended try_wait was
+// seen to resume several hundred cycles after the phase completed; a poll costs one issue
+// slot every few tens of cycles while it waits.
+__device__ __forceinline__ bool mbar_spin(const Ctx& c, uint32_t bar, uint32_t parity, int site) {
+  if (mbar_test_wait(bar, parity)) return true;
+  long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_test_wait(bar, parity)) return true;
+    if (*c.abort_smem) return false;
+    if (clock64() - t0 > kTimeoutCycles) { signal_abort(c, site); return false; }
+  }
+}
+__device__ __forceinline__ bool warp_spin(const Ctx& c, uint32_t bar, uint32_t parity, int site) {
+  return __all_sync(0xffffffffu, mbar_spin(c, bar, parity, site));
 }
 
 template <int BLOCK, int D>
@@ -350,28 +383,34 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
   const uint32_t bar0 = sbase + G::OFF_BAR;
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-  constexpr int B_TASK_FULL = 0, B_TASK_EMPTY = 2, B_Q_FULL = 4, B_Q_EMPTY = 5, B_KV_FULL = 6,
-                B_KV_EMPTY = 6 + G::NSTAGE, B_S_FULL = 6 + 2 * G::NSTAGE, B_P_FULL = B_S_FULL + G::NSBUF,
-                B_PV_DONE = B_P_FULL + G::NSBUF, B_O_FULL = B_PV_DONE + 1, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1;
-  static_assert(B_FINAL + 1 <= G::N_BAR, "barrier count");
+  constexpr int B_TASK_FULL = 0, B_TASK_EMPTY = 2, B_Q_FULL = 4, B_Q_EMPTY = 5, B_K_FULL = 6,
+                B_K_EMPTY = B_K_FULL + G::NKS, B_V_FULL = B_K_EMPTY + G::NKS, B_V_EMPTY = B_V_FULL + G::NVS,
+                B_S_FULL = B_V_EMPTY + G::NVS, B_P_FULL = B_S_FULL + G::NSBUF, B_S_FREE = B_P_FULL + G::NSBUF,
+                B_O_FULL = B_S_FREE + G::NSBUF, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1, B_MX = B_FINAL + 1;
+  static_assert(B_MX + 8 <= G::N_BAR, "barrier count");
   Task* tasks = reinterpret_cast<Task*>(smem + G::OFF_TASK);
-  float* mx = reinterpret_cast<float*>(smem + G::OFF_MX);            // [2][2][128] row-max / row-sum exchange
+  volatile float* mpub = reinterpret_cast<volatile float*>(smem + G::OFF_MX);   // [block parity][128] reference max after a block
+  float2* ex = reinterpret_cast<float2*>(smem + G::OFF_MX + 2 * 128 * 4);       // [task parity][team][128] (reference, sum)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + G::OFF_MISC);
   volatile int* abort_smem = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 4);
   Ctx ctx{bar0, abort_smem, p.ws, p.dev_status};
 
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_TASK_FULL + i), 1); mbar_init(BAR(B_TASK_EMPTY + i), 9); }
+    // a task is read by the two MMA issuers and the eight softmax warps
+    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_TASK_FULL + i), 1); mbar_init(BAR(B_TASK_EMPTY + i), 10); }
     mbar_init(BAR(B_Q_FULL), 1);
     mbar_init(BAR(B_Q_EMPTY), 1);
-    for (int i = 0; i < G::NSTAGE; ++i) { mbar_init(BAR(B_KV_FULL + i), 1); mbar_init(BAR(B_KV_EMPTY + i), 1); }
-    for (int i = 0; i < G::NSBUF; ++i) mbar_init(BAR(B_S_FULL + i), 1);
-    // one P barrier per S buffer: a warp may run up to two blocks ahead of the slowest one
-    for (int i = 0; i < G::NSBUF; ++i) mbar_init(BAR(B_P_FULL + i), 8);
-    mbar_init(BAR(B_PV_DONE), 1);
+    for (int i = 0; i < G::NKS; ++i) { mbar_init(BAR(B_K_FULL + i), 1); mbar_init(BAR(B_K_EMPTY + i), 1); }
+    for (int i = 0; i < G::NVS; ++i) { mbar_init(BAR(B_V_FULL + i), 1); mbar_init(BAR(B_V_EMPTY + i), 1); }
+    for (int i = 0; i < G::NSBUF; ++i) {
+      mbar_init(BAR(B_S_FULL + i), 1);
+      mbar_init(BAR(B_P_FULL + i), 4);     // the four warps of the team that owns the block
+      mbar_init(BAR(B_S_FREE + i), 1);
+    }
     mbar_init(BAR(B_O_FULL), 1);
     mbar_init(BAR(B_O_FREE), 8);
     mbar_init(BAR(B_FINAL), 1);
+    for (int i = 0; i < 8; ++i) mbar_init(BAR(B_MX + i), 1);
     *abort_smem = 0;
     fence_mbar_init();
     fence_proxy_async();
@@ -379,22 +418,24 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   // the MMA reads all 128 rows of the Q region even when a query block has 64 rows: clear it once
   for (int i = tid; i < G::Q_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(smem + G::OFF_Q)[i] = make_uint4(0, 0, 0, 0);
   fence_proxy_async();
-  if (warp == 1) {
+  if (warp == kPvWarp) {
     tmem_alloc(smem_u32(tmem_holder), G::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *tmem_holder;
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_holder, 0);
 
-  if (warp == 0) {
+  // Every role walks the same sequence of tasks (query blocks) and, inside a task, of KV blocks;
+  // block number g (counted over the CTA's whole life) uses S buffer g mod 3, K stage g mod NKS
+  // and V stage g mod NVS, so no role needs to be told where a tile or a buffer is.
+  if (warp == kProducerWarp) {
     // ============================================================== producer
     if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); }
-    uint32_t task_it = 0, q_it = 0, kv_it = 0;
-    TRACE_DECL;
+    uint32_t task_it = 0, q_it = 0, k_it = 0, v_it = 0;
     bool ok = true;
-    uint32_t armed_mask = 0, armed_parity = 0;   // per stage: parity of the last load armed on it
+    uint32_t k_armed = 0, k_parity = 0, v_armed = 0, v_parity = 0;   // per stage: parity of the last load armed on it
     bool q_armed = false; uint32_t q_armed_parity = 0;
     while (ok) {
       long long t = 0;
@@ -435,7 +476,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
       q_armed = true; q_armed_parity = q_it & 1;
       ++q_it;
-      // K/V tiles in the order the MMA warp consumes them: K_0..K_2, then V_j, K_{j+3} for each j
+      // K tiles run three blocks ahead of the V tiles, like the MMAs that consume them
       int chunk_base = -64, my_idx = 0;
       auto load_tile = [&](bool is_k, int j) -> bool {
         if (j < chunk_base || j >= chunk_base + 32) {
@@ -445,25 +486,26 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
         int blk = __shfl_sync(0xffffffffu, my_idx, j - chunk_base);
         if (blk < 0 || blk >= p.n_b) blk = 0;            // malformed list: stay in range
-        const uint32_t st = kv_it % G::NSTAGE, sph = (kv_it / G::NSTAGE) & 1;
-        if (!warp_wait(ctx, BAR(B_KV_EMPTY + st), sph ^ 1, 3)) return false;
-        TRACE(3, 20 + (is_k ? 0 : 1), j);
+        const uint32_t it = is_k ? k_it : v_it;
+        const uint32_t nst = is_k ? (uint32_t)G::NKS : (uint32_t)G::NVS;
+        const uint32_t st = it % nst, sph = (it / nst) & 1;
+        const int b_full = (is_k ? B_K_FULL : B_V_FULL) + (int)st, b_empty = (is_k ? B_K_EMPTY : B_V_EMPTY) + (int)st;
+        if (!warp_wait(ctx, BAR(b_empty), sph ^ 1, 3)) return false;
         if (lane == 0) {
 #ifdef WAVEAL_DBG_NOLOAD
-          if (kv_it >= (uint32_t)G::NSTAGE) { mbar_arrive(BAR(B_KV_FULL + st)); } else
+          if (it >= nst) { mbar_arrive(BAR(b_full)); } else
 #endif
           {
-          mbar_expect_tx(BAR(B_KV_FULL + st), G::TILE_BYTES);
+          mbar_expect_tx(BAR(b_full), G::TILE_BYTES);
           const CUtensorMap* tm = is_k ? &tmK : &tmV;
+          const uint32_t dst = sbase + (is_k ? G::OFF_K : G::OFF_V) + st * G::TILE_BYTES;
 #pragma unroll
           for (int s = 0; s < G::SLABS; ++s)
-            tma_load_3d(sbase + G::OFF_KV + st * G::TILE_BYTES + s * G::KV_SLAB_BYTES, tm, s * 64, blk * G::BK, tk.h,
-                        BAR(B_KV_FULL + st));
+            tma_load_3d(dst + s * G::KV_SLAB_BYTES, tm, s * 64, blk * G::BK, tk.h, BAR(b_full));
           }
         }
-        armed_mask |= 1u << st;
-        armed_parity = (armed_parity & ~(1u << st)) | (sph << st);
-        ++kv_it;
+        if (is_k) { k_armed |= 1u << st; k_parity = (k_parity & ~(1u << st)) | (sph << st); ++k_it; }
+        else { v_armed |= 1u << st; v_parity = (v_parity & ~(1u << st)) | (sph << st); ++v_it; }
         return true;
       };
       for (int j = 0; j < G::NSBUF && j < tk.n && ok; ++j) ok = load_tile(true, j);
@@ -474,30 +516,34 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
     if (*abort_smem) {
       // leave no bulk copy in flight into this CTA's shared memory (bounded)
-      for (int st = 0; st < G::NSTAGE; ++st)
-        if (armed_mask & (1u << st)) {
+      for (int st = 0; st < G::NKS; ++st)
+        if (k_armed & (1u << st)) {
           long long t0 = clock64();
-          while (!mbar_try_wait(BAR(B_KV_FULL + st), (armed_parity >> st) & 1) && clock64() - t0 < kTimeoutCycles / 4) {}
+          while (!mbar_try_wait(BAR(B_K_FULL + st), (k_parity >> st) & 1) && clock64() - t0 < kTimeoutCycles / 4) {}
+        }
+      for (int st = 0; st < G::NVS; ++st)
+        if (v_armed & (1u << st)) {
+          long long t0 = clock64();
+          while (!mbar_try_wait(BAR(B_V_FULL + st), (v_parity >> st) & 1) && clock64() - t0 < kTimeoutCycles / 4) {}
         }
       if (q_armed) {
         long long t0 = clock64();
         while (!mbar_try_wait(BAR(B_Q_FULL), q_armed_parity) && clock64() - t0 < kTimeoutCycles / 4) {}
       }
     }
-  } else if (warp == 1) {
-    // ============================================================== MMA issuer
-    // Every operand of a tcgen05 instruction (descriptors, tensor-memory addresses, barrier
-    // addresses) must stay warp-uniform in the compiler's eyes, otherwise each MMA pays for
-    // moves into uniform registers and the issue rate drops below the tensor pipe's: values
-    // read from shared memory are broadcast with a shuffle, ring positions are advanced by
-    // compare-and-reset instead of modulo.
+  } else if (warp == kQkWarp) {
+    // ============================================================== MMA issuer 1: S = Q K^T
+    // Two warps issue the MMAs, one per product: the bookkeeping of each (barrier waits, ring
+    // arithmetic, descriptor set-up: a few hundred cycles of dependent scalar work per block)
+    // then runs while the other's MMAs execute, and the tensor pipe is not left waiting for
+    // it.  MMAs of different threads are ordered through completion barriers only.
+    // Every operand of a tcgen05 instruction stays warp-uniform in the compiler's eyes
+    // (shuffle-broadcast values, compare-and-reset ring positions).
     constexpr uint32_t IDESC_QK = make_idesc(128, G::BK, false);
-    constexpr uint32_t IDESC_PV = make_idesc(128, D, true);
-    uint32_t task_slot = 0, task_ph = 0, q_ph = 0, o_ph = 1, kv_st = 0, kv_ph = 0, p_phase = 0;
+    uint32_t task_slot = 0, task_ph = 0, q_ph = 0, k_st = 0, k_ph = 0, sb = 0, free_bits = 0, first_uses = G::NSBUF;
     TRACE_DECL;
     const uint64_t qdesc0 = make_desc(sbase + G::OFF_Q, 16, 1024);
-    const uint64_t kdesc0 = make_desc(sbase + G::OFF_KV, 16, 1024);
-    const uint64_t vdesc0 = make_desc(sbase + G::OFF_KV, G::KV_SLAB_BYTES, 1024);
+    const uint64_t kdesc0 = make_desc(sbase + G::OFF_K, 16, 1024);
     bool ok = true;
     while (ok) {
       ok = warp_wait(ctx, BAR(B_TASK_FULL + task_slot), task_ph, 10);
@@ -512,14 +558,23 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       ok = warp_wait(ctx, BAR(B_Q_FULL), q_ph, 11);
       if (!ok) break;
       q_ph ^= 1;
-      // S[sb] = Q K_j^T (sb = j mod 3); overwrites the P tile that aliases S[sb], which the
-      // P V three blocks earlier (issued before by this warp, executed in order) has consumed.
-      // The caller has already waited for the K tile in stage kv_st.
-      auto issue_qk = [&](uint32_t sb) {
-        TRACE(0, 4, (int)kv_st);
+      for (int j = 0; j < n && ok; ++j) {
+        ok = warp_spin(ctx, BAR(B_K_FULL + k_st), k_ph, 12);
+        if (!ok) break;
+        // S[sb] also holds the P tile of the block that used it last: wait until that block's
+        // P V has completed (its commit is phase number uses-1 of the buffer's barrier)
+        if (first_uses > 0) {
+          --first_uses;
+        } else {
+          ok = warp_spin(ctx, BAR(B_S_FREE + sb), ((free_bits >> sb) & 1u) ^ 1u, 13);
+          if (!ok) break;
+        }
+        free_bits ^= 1u << sb;
+        TRACE(3, 4, j);
+        tc_fence_after();
         {
           // descriptors differ from the per-kernel bases only in the 14-bit address field
-          const uint64_t kd = kdesc0 + (uint64_t)(kv_st * (uint32_t)(G::TILE_BYTES >> 4));
+          const uint64_t kd = kdesc0 + (uint64_t)(k_st * (uint32_t)(G::TILE_BYTES >> 4));
           const uint32_t d_s = tmem_base + sb * G::S_STRIDE;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
@@ -528,45 +583,49 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                       kd + (uint64_t)(((k / 4) * G::KV_SLAB_BYTES + (k % 4) * 32) >> 4), IDESC_QK, k > 0);
 #endif
           }
-          tc_commit(BAR(B_KV_EMPTY + kv_st));
+          tc_commit(BAR(B_K_EMPTY + k_st));
           tc_commit(BAR(B_S_FULL + sb));
+          if (j == n - 1) tc_commit(BAR(B_Q_EMPTY));
         }
-        TRACE(0, 5, (int)kv_st);
-        if (++kv_st == (uint32_t)G::NSTAGE) { kv_st = 0; kv_ph ^= 1; }
-      };
-      for (int j = 0; j < G::NSBUF && j < n && ok; ++j) {
-        ok = warp_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, 12);
-        if (ok) issue_qk((uint32_t)j);
+        TRACE(3, 5, j);
+        if (++k_st == (uint32_t)G::NKS) { k_st = 0; k_ph ^= 1; }
+        if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
+    }
+  } else if (warp == kPvWarp) {
+    // ============================================================== MMA issuer 2: O += P V
+    constexpr uint32_t IDESC_PV = make_idesc(128, D, true);
+    uint32_t task_slot = 0, task_ph = 0, o_ph = 1, v_st = 0, v_ph = 0, sb = 0, p_phase = 0;
+    TRACE_DECL;
+    const uint64_t vdesc0 = make_desc(sbase + G::OFF_V, G::KV_SLAB_BYTES, 1024);
+    bool ok = true;
+    while (ok) {
+      ok = warp_wait(ctx, BAR(B_TASK_FULL + task_slot), task_ph, 10);
       if (!ok) break;
-      if (n <= G::NSBUF) tc_commit(BAR(B_Q_EMPTY));
+      const int n = __shfl_sync(0xffffffffu, tasks[task_slot].n, 0);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + task_slot));
+      task_slot ^= 1;
+      task_ph ^= (task_slot == 0);
+      if (n < 0) break;
+      if (n == 0) continue;
       // the output accumulator of the previous task has been read by the epilogue
       ok = warp_wait(ctx, BAR(B_O_FREE), o_ph, 16);
       if (!ok) break;
       o_ph ^= 1;
-      // answers for the first P V of the task
-      uint32_t tok_p = mbar_test_wait(BAR(B_P_FULL + 0), p_phase & 1u);
-      uint32_t tok_v = mbar_test_wait(BAR(B_KV_FULL + kv_st), kv_ph);
-      uint32_t sb = 0;
       for (int j = 0; j < n && ok; ++j) {
-        // O (+)= P_j V_j, P_j read from tensor memory
-        ok = finish_wait(ctx, BAR(B_P_FULL + sb), (p_phase >> sb) & 1u, tok_p, 14);
+        ok = warp_spin(ctx, BAR(B_P_FULL + sb), (p_phase >> sb) & 1u, 14);
         if (!ok) break;
         p_phase ^= 1u << sb;
         TRACE(0, 1, j);
-        ok = finish_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, tok_v, 15);
+        ok = warp_spin(ctx, BAR(B_V_FULL + v_st), v_ph, 15);
         if (!ok) break;
         TRACE(0, 2, j);
-        const bool more_qk = j + G::NSBUF < n;
-        // the K tile of block j+3 sits in the stage after this V tile: ask now, use after the MMAs
-        uint32_t k_st = kv_st + 1, k_ph = kv_ph;
-        if (k_st == (uint32_t)G::NSTAGE) { k_st = 0; k_ph ^= 1; }
-        uint32_t tok_k = more_qk ? mbar_test_wait(BAR(B_KV_FULL + k_st), k_ph) : 1u;
         tc_fence_after();
         {
           // V tile as the N x K operand with N (head_dim) contiguous: 8 keys per 1024-byte
           // group along K (16 keys = 2048 bytes per MMA), next 64 columns of head_dim one slab further
-          const uint64_t vd = vdesc0 + (uint64_t)(kv_st * (uint32_t)(G::TILE_BYTES >> 4));
+          const uint64_t vd = vdesc0 + (uint64_t)(v_st * (uint32_t)(G::TILE_BYTES >> 4));
           const uint32_t pbase = tmem_base + sb * G::S_STRIDE;
           const uint32_t d_o = tmem_base + G::O_COL;
           if (j > 0) {
@@ -584,32 +643,17 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #endif
             }
           }
-          tc_commit(BAR(B_KV_EMPTY + kv_st));
-          tc_commit(BAR(B_PV_DONE));
+          tc_commit(BAR(B_V_EMPTY + v_st));
+          tc_commit(BAR(B_S_FREE + sb));
           if (j == n - 1) tc_commit(BAR(B_O_FULL));
         }
         TRACE(0, 3, j);
-        if (++kv_st == (uint32_t)G::NSTAGE) { kv_st = 0; kv_ph ^= 1; }
-        if (more_qk) {
-          ok = finish_wait(ctx, BAR(B_KV_FULL + kv_st), kv_ph, tok_k, 12);
-          if (!ok) break;
-        }
-        // answers for the next P V (its V tile follows the K tile just checked)
-        if (j + 1 < n) {
-          uint32_t v_st = kv_st, v_ph = kv_ph;
-          if (more_qk) { if (++v_st == (uint32_t)G::NSTAGE) { v_st = 0; v_ph ^= 1; } }
-          const uint32_t nsb = (sb + 1 == (uint32_t)G::NSBUF) ? 0u : sb + 1;
-          tok_p = mbar_test_wait(BAR(B_P_FULL + nsb), (p_phase >> nsb) & 1u);
-          tok_v = mbar_test_wait(BAR(B_KV_FULL + v_st), v_ph);
-        }
-        if (more_qk) {
-          issue_qk(sb);
-          if (j + G::NSBUF == n - 1) tc_commit(BAR(B_Q_EMPTY));
-        }
+        if (++v_st == (uint32_t)G::NVS) { v_st = 0; v_ph ^= 1; }
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
     }
-    // every MMA issued by this warp has completed before tensor memory is released
+    // every MMA has completed before tensor memory is released: the last P V depends on all
+    // the Q K^T products through the softmax warps
     tc_commit(BAR(B_FINAL));
     __syncwarp();
     {
@@ -618,16 +662,22 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
   } else {
     // ============================================================== softmax / epilogue
-    // All eight warps work on every block: thread (row, half) owns half a row of S, so two
-    // warps per scheduler interleave and hide each other's latencies; the two halves of a row
-    // exchange their maxima through shared memory (one 64-thread named barrier per block).
+    // Two teams of four warps take the KV blocks of a task in turn (team = block index mod 2);
+    // a thread owns one whole row of S for its team's blocks.  On every scheduler sits one warp
+    // of each team, half a block apart in time: while one is in its exponentials (bound by the
+    // transcendental unit) the other waits for S, loads it, takes the row max and stores P, so
+    // the latencies of one team hide behind the arithmetic of the other.  Nothing is exchanged
+    // inside a row; the teams only hand the running reference max of each row to each other
+    // (shared memory + one mbarrier per lane quadrant and block parity), because both
+    // accumulate into the same O.  Each team keeps the sum of its own blocks; the epilogue adds
+    // the two.
     const int sw = warp - kSoftmaxWarp0;       // 0..7
     const int quad = warp & 3;                 // tensor-memory lane quadrant this warp may access
-    const int half = sw >> 2;                  // which half of the S / O columns
+    const int team = sw >> 2;                  // owns blocks j with (j & 1) == team; epilogue: half of the O columns
     const int r = quad * 32 + lane;            // row of the 128-row MMA tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t o_addr = tmem_base + lane_addr + G::O_COL + half * G::CO;
-    uint32_t task_it = 0, s_phase = 0, o_it = 0, pv_total = 0, blk_it = 0;
+    const uint32_t o_row = tmem_base + lane_addr + G::O_COL;
+    uint32_t task_it = 0, s_phase = 0, o_it = 0, mx_phase = 0, sb = 0;   // s_phase bit b: parity of the uses of S[b] so far
     TRACE_DECL;
     bool ok = true;
     while (ok) {
@@ -637,142 +687,180 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const Task tk = tasks[slot];
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + slot));
+      float2* exb = ex + (task_it & 1) * 256;
       ++task_it;
       if (tk.n < 0) break;
       const long long q_tok = (long long)tk.row * G::BQ + r;
       const bool row_live = r < G::BQ && q_tok < p.seq_q;
-      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + half * G::CO;
+      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + team * G::CO;
       if (tk.n == 0) {
         if (row_live) {
 #pragma unroll
           for (int c = 0; c < G::CO / 8; ++c) reinterpret_cast<uint4*>(o_ptr)[c] = make_uint4(0, 0, 0, 0);
-          if (p.lse && half == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
+          if (p.lse && team == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
         }
         continue;
       }
-      float m_used = -INFINITY, l_run = 0.f;
-      uint32_t sb = 0;
+      // l_run: sum over this team's blocks, relative to the reference m_ref
+      float m_ref = -INFINITY, l_run = 0.f;
       for (int j = 0; j < tk.n && ok; ++j) {
-        ok = warp_wait(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
-        if (!ok) break;
-        s_phase ^= 1u << sb;
-        if (sw == 2 || sw == 6) TRACE(1 + half, 10 + half, j);
-        tc_fence_after();
-        const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE;
-        uint32_t sv[G::CS];
-        if constexpr (G::CS == 64) {
-          WAVEAL_TMEM_LD32(s_addr + half * 64, sv, 0);
-          WAVEAL_TMEM_LD32(s_addr + half * 64 + 32, sv, 32);
-          WAVEAL_TMEM_WAIT_LD32(sv, 0);
-          WAVEAL_TMEM_WAIT_LD32(sv, 32);
-        } else {
-          WAVEAL_TMEM_LD32(s_addr + half * 32, sv, 0);
-          WAVEAL_TMEM_WAIT_LD32(sv, 0);
-        }
-        if (sw == 2 || sw == 6) TRACE(1 + half, 12 + half, j);
-        // scores of keys beyond seq_kv (ragged last block) do not exist
-        if (j == tk.n - 1 && tk.tail_valid < G::BK) {
-#pragma unroll
-          for (int c = 0; c < G::CS; ++c)
-            if (half * G::CS + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
-        }
-        // row max: eight independent chains, then the other half of the row through smem
-        float mx8[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(sv[i]);
-#pragma unroll
-        for (int c = 8; c < G::CS; c += 8) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(sv[c + i]));
-        }
-        const float mloc = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                                 fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-        float* mxb = mx + (blk_it & 1) * 256;
-        ++blk_it;
-        mxb[half * 128 + r] = mloc;
-        named_bar_sync(1 + quad, 64);
-        const float m_cand = fmaxf(m_used, fmaxf(mloc, mxb[(half ^ 1) * 128 + r]) * p.sl2);
-        // keep the stale reference max unless it is exceeded by more than 2^8 (exact: the
-        // final normalisation divides by a sum taken with the same reference); both halves of a
-        // row see the same numbers and the two warps hold the same rows, so they decide alike
-        const bool grow = __any_sync(0xffffffffu, m_cand > m_used + 8.0f);
-        float alpha = 1.f;
-        if (grow) {
-          alpha = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_cand);
-          m_used = m_cand;
-          l_run *= alpha;
-        }
-        uint32_t pk[G::PC];
-        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-        // p' = 2^(s*scale*log2e - m + log2(1 + 2^-9)); P is p' cut to its top 16 bits (one byte
-        // permute per pair instead of a conversion on the transcendental pipe).  The extra
-        // factor centres the cut's error around zero, and the row sum adds the SAME cut values
-        // the tensor core multiplies with, so numerator and denominator stay consistent.
-        const float neg_m = ((m_used == -INFINITY) ? 0.f : -m_used) + 0.0028150156f;
-#pragma unroll
-        for (int c = 0; c < G::CS; c += 2) {
-          const float x0 = fmaf(__uint_as_float(sv[c]), p.sl2, neg_m);
-          const float x1 = fmaf(__uint_as_float(sv[c + 1]), p.sl2, neg_m);
-          // every kPolyEvery-th pair takes the polynomial path (a fixed pattern per column, so
-          // the result of a row does not depend on the execution order)
-          const bool poly = kPolyEvery > 0 && ((c >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == (kPolyEvery - 1);
-          const uint32_t b0 = __float_as_uint(poly ? ex2_fma(x0) : ex2(x0));
-          const uint32_t b1 = __float_as_uint(poly ? ex2_fma(x1) : ex2(x1));
-          ls4[(c >> 1) & 3] += __uint_as_float(b0 & 0xFFFF0000u) + __uint_as_float(b1 & 0xFFFF0000u);
-          pk[c / 2] = __byte_perm(b0, b1, 0x7632);
-        }
-        l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-        if (sw == 2 || sw == 6) TRACE(1 + half, 14 + half, j);
-        // rare: the reference grew, so the accumulated O is rescaled; P_{j-1} V_{j-1} (the last MMA
-        // that touches O) must be complete - the barrier has seen exactly pv_total + j - 1 or
-        // pv_total + j phases by now, so a parity wait is unambiguous
-        if (grow && j > 0) {
-          ok = warp_wait(ctx, BAR(B_PV_DONE), (pv_total + (uint32_t)j - 1u) & 1u, 22);
+        const uint32_t par = (uint32_t)j & 1u;
+        if ((int)par == team) {
+          ok = warp_spin(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
           if (!ok) break;
+          if (quad == 2) TRACE(1 + team, 10 + team, j);
           tc_fence_after();
+          const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE;
+          const bool ragged = j == tk.n - 1 && tk.tail_valid < G::BK;
+#ifndef WAVEAL_DBG_NOSM   // (timing experiments only: with the macro the softmax warps just pass the barriers on)
+          // ---- pass 1: row max (the values are loaded again for the exponentials: a second
+          // tensor-memory load is cheaper than 128 live registers)
+          float mloc = -INFINITY;
 #pragma unroll
-          for (int c0 = 0; c0 < G::CO; c0 += 32) {
-            uint32_t ov[32];
-            WAVEAL_TMEM_LD32(o_addr + c0, ov, 0);
-            WAVEAL_TMEM_WAIT_LD32(ov, 0);
+          for (int ch = 0; ch < G::NCH; ++ch) {
+            uint32_t sv[G::CH];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-            WAVEAL_TMEM_ST32(o_addr + c0, ov, 0);
+            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_LD32(s_addr + ch * G::CH + c, sv, c);
+#pragma unroll
+            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_WAIT_LD32(sv, c);
+            // scores of keys beyond seq_kv (ragged last block) do not exist
+            if (ragged) {
+#pragma unroll
+              for (int c = 0; c < G::CH; ++c)
+                if (ch * G::CH + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
+            }
+            float mx8[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(sv[i]);
+#pragma unroll
+            for (int c = 8; c < G::CH; c += 8) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(sv[c + i]));
+            }
+            mloc = fmaxf(mloc, fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                                     fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7]))));
           }
+          if (quad == 2) TRACE(1 + team, 12 + team, j);
+          // ---- the row's reference after block j-1, from the other team
+          float m_prev = -INFINITY;
+          if (j > 0) {
+            // that team's arrival for block j-1 is phase number (blocks of that parity so far) - 1
+            ok = warp_spin(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24);
+            if (!ok) break;
+            m_prev = mpub[(par ^ 1u) * 128 + r];
+          }
+          const float m_cand = fmaxf(m_prev, mloc * p.sl2);
+          // keep the stale reference unless it is exceeded by more than 2^8 (exact: the final
+          // normalisation divides by a sum taken with the same reference)
+          const bool grow = __any_sync(0xffffffffu, m_cand > m_prev + 8.0f);
+          const float m_new = grow ? m_cand : m_prev;
+          mpub[par * 128 + r] = m_new;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(BAR(B_MX + quad * 2 + par));
+          if (m_new != m_ref) {
+            l_run *= (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
+            m_ref = m_new;
+          }
+          // p' = 2^(s*scale*log2e - m + log2(1 + 2^-9)); P is p' cut to its top 16 bits (one byte
+          // permute per pair instead of a conversion).  The extra factor centres the cut's error
+          // around zero, like a rounding; the row sum adds the uncut p' and the epilogue takes
+          // the factor out again.  Multiply-adds and sums work on register pairs (f32x2).
+          const float neg_m = ((m_new == -INFINITY) ? 0.f : -m_new) + 0.0028150156f;
+          float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+          // ---- pass 2: exponentials; P_j (bf16 pairs) goes over the first half of the row's own
+          // S columns, each chunk after its S values have been read
+#pragma unroll
+          for (int ch = 0; ch < G::NCH; ++ch) {
+            uint32_t sv[G::CH];
+#pragma unroll
+            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_LD32(s_addr + ch * G::CH + c, sv, c);
+#pragma unroll
+            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_WAIT_LD32(sv, c);
+            if (ragged) {
+#pragma unroll
+              for (int c = 0; c < G::CH; ++c)
+                if (ch * G::CH + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
+            }
+            uint32_t pk[G::CH / 2];
+#pragma unroll
+            for (int c = 0; c < G::CH; c += 2) {
+              float x0, x1;
+              ffma2(x0, x1, __uint_as_float(sv[c]), __uint_as_float(sv[c + 1]), p.sl2, p.sl2, neg_m, neg_m);
+              float e0, e1;
+              if (kPolyEvery > 0 && ((c >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == (kPolyEvery > 0 ? kPolyEvery : 1) - 1) {
+                ex2_fma2(e0, e1, x0, x1);
+              } else {
+                e0 = ex2(x0); e1 = ex2(x1);
+              }
+              fadd2(ls4[c & 2], ls4[(c & 2) + 1], ls4[c & 2], ls4[(c & 2) + 1], e0, e1);
+              pk[c / 2] = __byte_perm(__float_as_uint(e0), __float_as_uint(e1), 0x7632);
+            }
+            if constexpr (G::CH == 64) { WAVEAL_TMEM_ST32(s_addr + ch * 32, pk, 0); }
+            else { WAVEAL_TMEM_ST16(s_addr + ch * 16, pk, 0); }
+          }
+          l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+          if (quad == 2) TRACE(1 + team, 14 + team, j);
+          // rare: the reference grew, so O (blocks 0..j-1) is rescaled; its last MMA (block j-1)
+          // must be complete: that is the latest phase of the barrier of the S buffer before
+          // this one (the next P V on that buffer needs a P this team has not produced yet)
+          if (grow && j > 0) {
+            const uint32_t sbp = sb == 0 ? (uint32_t)G::NSBUF - 1u : sb - 1u;
+            ok = warp_wait(ctx, BAR(B_S_FREE + sbp), ((s_phase >> sbp) & 1u) ^ 1u, 22);
+            if (!ok) break;
+            tc_fence_after();
+            const float alpha = ex2(m_prev - m_new);
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+              uint32_t ov[32];
+              WAVEAL_TMEM_LD32(o_row + c0, ov, 0);
+              WAVEAL_TMEM_WAIT_LD32(ov, 0);
+#pragma unroll
+              for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+              WAVEAL_TMEM_ST32(o_row + c0, ov, 0);
+            }
+          }
+#else
+          if (j > 0) { ok = warp_spin(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24); if (!ok) break; }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(BAR(B_MX + quad * 2 + par));
+          l_run = 1.f; m_ref = 0.f;
+#endif
+          tc_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb));
+          if (quad == 2) TRACE(1 + team, 16 + team, j);
         }
-        // P_j (bf16 pairs) over the first half of the columns of S[sb]
-        if constexpr (G::PC == 32) { WAVEAL_TMEM_ST32(s_addr + half * 32, pk, 0); }
-        else { WAVEAL_TMEM_ST16(s_addr + half * 16, pk, 0); }
-        tc_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb));
-        if (sw == 2 || sw == 6) TRACE(1 + half, 16 + half, j);
+        // both teams count every block
+        s_phase ^= 1u << sb;
+        mx_phase ^= 1u << par;
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
       if (!ok) break;
-      pv_total += (uint32_t)tk.n;
-      // ---- epilogue: O / l at the original row position
+      // ---- epilogue: O / l at the original row position; l = the two teams' sums brought to
+      // the final reference (the larger of the two, references never shrink)
       ok = warp_wait(ctx, BAR(B_O_FULL), o_it & 1, 23);
       if (!ok) break;
       ++o_it;
       tc_fence_after();
-      if (sw == 2 || sw == 6) TRACE(1 + half, 18 + half, tk.n);
-      float* lx = mx + (blk_it & 1) * 256;      // the buffer the last block did not use
-      ++blk_it;
-      lx[half * 128 + r] = l_run;
+      if (quad == 2) TRACE(1 + team, 18 + team, tk.n);
+      exb[team * 128 + r] = make_float2(m_ref, l_run);
       named_bar_sync(1 + quad, 64);
-      const float l_tot = l_run + lx[(half ^ 1) * 128 + r];
-      const float inv_l = 1.0f / l_tot;
+      const float2 oth = exb[(team ^ 1) * 128 + r];
+      const float m_all = fmaxf(m_ref, oth.x);
+      const float a_self = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_all);
+      const float a_oth = (oth.x == -INFINITY) ? 0.f : ex2(oth.x - m_all);
+      const float l_tot = a_self * l_run + a_oth * oth.y;
+      const float inv_l = 1.0019531f / l_tot;    // the sums carry the centring factor 1 + 2^-9
       uint32_t ov[G::CO];
 #pragma unroll
-      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(o_addr + c, ov, c);
+      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(o_row + team * G::CO + c, ov, c);
 #pragma unroll
       for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(ov, c);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_O_FREE));
-      if (sw == 2 || sw == 6) TRACE(1 + half, 30 + half, tk.n);
+      if (quad == 2) TRACE(1 + team, 30 + team, tk.n);
       if (row_live) {
 #pragma unroll
         for (int c = 0; c < G::CO; c += 8) {
@@ -785,7 +873,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           }
           *reinterpret_cast<uint4*>(o_ptr + c) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (p.lse && half == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_used + log2f(l_tot)) * 0.6931471805599453f;
+        if (p.lse && team == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_all + log2f(l_tot) - 0.0028150156f) * 0.6931471805599453f;
       }
     }
   }
@@ -793,7 +881,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kPvWarp) {
     tc_fence_after();
     tmem_dealloc(tmem_base, G::TMEM_COLS);
   }
