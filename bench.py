@@ -175,7 +175,14 @@ def run_waveal(args, cfg):
     H, S, Sp, D, B = cfg.heads, cfg.seq, cfg.seq_pad, cfg.head_dim, cfg.block
     nb = cfg.n_blocks
     # ---- synthetic batch element of this rank: host (pinned) and device copies
-    masks = [I.make_mask(cfg, h) for h in range(H)]
+    if args.mask == "random20":
+        # the unstructured mask of the paper's Table 1 (20 % uniform columns per row): the locality floor
+        masks = [I.random_mask(nb, nb, 0.20, cfg.mask_seed * 1000 + h) for h in range(H)]
+    elif args.mask == "dense":
+        # all block pairs: the dense run behind the gap metric (1/density) / (t_dense / t_sparse)
+        masks = [np.ones((nb, nb), dtype=bool) for _ in range(H)]
+    else:
+        masks = [I.make_mask(cfg, h) for h in range(H)]
     bitmap_h = torch.from_numpy(np.stack([I.mask_to_bitmap(m) for m in masks]).view(np.int64)).pin_memory()
     ptr_np, idx_np = I.masks_to_csr(masks)
     pairs = int(ptr_np[-1])
@@ -197,7 +204,7 @@ def run_waveal(args, cfg):
                                  seed=cfg.plan_seed, kv_bytes_per_head=2 * Sp * D * 2)
     pws = torch.empty((wb.plan_workspace_bytes(pdesc) + 256,), dtype=torch.uint8, device=dev)
     aws = torch.empty((256,), dtype=torch.uint8, device=dev)
-    adesc = wb.attn_desc(q, k, v, o, S, S, B)
+    adesc = wb.attn_desc(q, k, v, o, S, S, B, args.head_order == "interleaved")
     status = torch.zeros((4,), dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
     launches = {"n": 0}
@@ -319,12 +326,14 @@ def run_waveal(args, cfg):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "heads": H, "head_dim": D, "seq": S, "block": B, "block_pairs": pairs,
                    "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode,
+                   "mask": args.mask, "head_order": args.head_order,
                    "step": "plan + attention", "l2": "inputs (Q,K,V,O %.1f GB) larger than L2, no flush" %
                    (4 * H * Sp * D * 2 / 1e9), "batch_elements": world},
         "roofline": {"bound": "tensor", "kernel": "k_bsattn_fwd", "achieved": achieved, "peak": pk["bf16"],
                      "unit": "TFLOP/s", "frac": achieved / pk["bf16"], "peak_source": pk["source"] + " (burst)",
                      "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
-                     "kernel_ms": attn_ms, "traffic": ncu_traffic(cfg.name)},
+                     "kernel_ms": attn_ms,
+                     "traffic": ncu_traffic(cfg.name) if args.mask == "videomask" else None},
         "kernel": {"attn_ms_reordered": t_reo, "attn_ms_natural": t_nat, "speedup_vs_natural": t_nat / t_reo,
                    "tflops_reordered": flops / t_reo / 1e9, "tflops_natural": flops / t_nat / 1e9,
                    "plan_ms": t_plan, "plan_ms_auto": t_plan_auto, "auto_skipped_heads": skipped,
@@ -353,6 +362,11 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling / parity cases)")
     ap.add_argument("--plan-mode", default="reorder", choices=["reorder", "natural", "auto", "stage1", "stage2"],
                     help="which stages the plan of the timed step runs (Section 6.5 ablation); the headline is 'reorder'")
+    ap.add_argument("--mask", default="videomask", choices=["videomask", "random20", "dense"],
+                    help="mask generator: the config's structured recipe, 20 %% uniform columns per row "
+                         "(the paper's Random row), or all pairs (dense run for the gap metric)")
+    ap.add_argument("--head-order", default="sequential", choices=["sequential", "interleaved"],
+                    help="ticket order: all rows of a head before the next head, or position-major over heads")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
