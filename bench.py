@@ -112,7 +112,7 @@ def oracle_sample(cfg, target_s=12.0, n_heads=4):
     for h in heads:
         mk = I.make_mask(cfg, h)
         t0 = time.perf_counter()
-        wo.plan_head(mk, 148, 10, cfg.plan_seed, h, mode=wo.MODE_FORCE_REORDER)
+        wo.plan_head(mk, 148, 5, cfg.plan_seed, h, mode=wo.MODE_FORCE_REORDER)   # T = the library default
         t_plan += time.perf_counter() - t0
         bits = [I.make_head_tensor(cfg, w, h).view(torch.int16).numpy().view(np.uint16) for w in "qkv"]
         data.append((mk, bits, rng.permutation(cfg.n_blocks)))
@@ -202,6 +202,8 @@ def run_waveal(args, cfg):
                  "stage1": wb.STAGE1_ONLY, "stage2": wb.STAGE2_ONLY}[args.plan_mode]
     pdesc = wb.plan_desc_default(heads=H, n_q_blocks=nb, n_kv_blocks=nb, wave_size=W, mode=step_mode,
                                  seed=cfg.plan_seed, kv_bytes_per_head=2 * Sp * D * 2)
+    if args.svd_iters > 0:
+        pdesc.svd_iters = args.svd_iters
     pws = torch.empty((wb.plan_workspace_bytes(pdesc) + 256,), dtype=torch.uint8, device=dev)
     aws = torch.empty((256,), dtype=torch.uint8, device=dev)
     adesc = wb.attn_desc(q, k, v, o, S, S, B, args.head_order == "interleaved")
@@ -297,6 +299,7 @@ def run_waveal(args, cfg):
         for g0, g1 in groups:
             gdesc[g0] = wb.plan_desc_default(heads=g1 - g0, n_q_blocks=nb, n_kv_blocks=nb, wave_size=W, mode=step_mode,
                                              seed=cfg.plan_seed, kv_bytes_per_head=2 * Sp * D * 2)
+            gdesc[g0].svd_iters = pdesc.svd_iters
 
         def e2e_step():
             start = ev()
@@ -359,7 +362,7 @@ def run_waveal(args, cfg):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "heads": H, "head_dim": D, "seq": S, "block": B, "block_pairs": pairs,
                    "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode,
-                   "mask": args.mask, "head_order": args.head_order,
+                   "mask": args.mask, "head_order": args.head_order, "svd_iters": int(pdesc.svd_iters),
                    "step": "plan + attention", "l2": "inputs (Q,K,V,O %.1f GB) larger than L2, no flush" %
                    (4 * H * Sp * D * 2 / 1e9), "batch_elements": world},
         "roofline": {"bound": "tensor", "kernel": "k_bsattn_fwd", "achieved": achieved, "peak": pk["bf16"],
@@ -400,6 +403,7 @@ def main():
                          "(the paper's Random row), or all pairs (dense run for the gap metric)")
     ap.add_argument("--head-order", default="sequential", choices=["sequential", "interleaved"],
                     help="ticket order: all rows of a head before the next head, or position-major over heads")
+    ap.add_argument("--svd-iters", type=int, default=0, help="T of Algorithm 1 (0 = the library default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

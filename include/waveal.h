@@ -66,7 +66,7 @@ typedef struct waveal_plan_desc {
   int32_t n_q_blocks;     /* M_B (Section 4.2)                                                */
   int32_t n_kv_blocks;    /* N_B                                                              */
   int32_t wave_size;      /* W = SMs x resident CTAs (Section 6.1); 0 = this device's SM count */
-  int32_t svd_iters;      /* T of Algorithm 1 (paper: 5-15)                                   */
+  int32_t svd_iters;      /* T of Algorithm 1 (paper: 5-15; library default 5)                */
   int32_t mode;           /* waveal_mode                                                      */
   uint64_t seed;          /* seed of the start block of Algorithm 1                           */
   /* guard thresholds, all integer comparisons (the "offline profile" of Section 4.5):       */

@@ -85,7 +85,7 @@ def test_plan_parity(name, frames, heads, wave):
     res = wb.plan_bitmap(d, _bitmap_dev(masks), debug=True)
     torch.cuda.synchronize()
     assert res.dev_status.tolist() == [0, 0, 0, 0]
-    exact = _check_plan(masks, hs, wave, 10, cfg.plan_seed, wo.MODE_FORCE_REORDER, res)
+    exact = _check_plan(masks, hs, wave, d.svd_iters, cfg.plan_seed, wo.MODE_FORCE_REORDER, res)
     assert exact >= 1          # fp64 on both sides: the permutation itself normally coincides
 
 
@@ -121,7 +121,7 @@ def test_guard_decisions_per_head():
     assert flags[0] == 0
     assert flags[1] == wo.FLAG_ALREADY_LOCAL | wo.FLAG_SKIPPED
     assert flags[2] & wo.FLAG_TOO_SPARSE and flags[2] & wo.FLAG_SKIPPED
-    _check_plan(masks, [0, 1, 2], 8, 10, 3, wo.MODE_AUTO, res, guard=guard)
+    _check_plan(masks, [0, 1, 2], 8, d.svd_iters, 3, wo.MODE_AUTO, res, guard=guard)
     # short-sequence case: the head's K+V fit the budget -> every head skipped
     d.kv_bytes_per_head, d.l2_bytes = 700, 3000
     res = wb.plan_bitmap(d, _bitmap_dev(masks), debug=True)
@@ -170,7 +170,7 @@ def test_plan_degenerate_and_rectangular(shape):
     d = wb.plan_desc_default(heads=3, n_q_blocks=m, n_kv_blocks=n, wave_size=wave, mode=wb.FORCE_REORDER, seed=2)
     res = wb.plan_bitmap(d, _bitmap_dev(masks), debug=True)
     torch.cuda.synchronize()
-    _check_plan(masks, [0, 1, 2], wave, 10, 2, wo.MODE_FORCE_REORDER, res)
+    _check_plan(masks, [0, 1, 2], wave, d.svd_iters, 2, wo.MODE_FORCE_REORDER, res)
     # all-ones / identical rows: centred mask is zero -> natural order
     assert np.array_equal(_np(res.order1[0]), np.arange(m))
     assert np.array_equal(_np(res.order1[2]), np.arange(m))
