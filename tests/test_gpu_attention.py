@@ -176,3 +176,36 @@ def test_full_size_sampled_parity_and_invariance(name):
                                             1 / math.sqrt(cfg.head_dim))
             errs.append(error_stats(o[h, lo:hi].float().cpu().numpy(), ref))
     assert max(e[0] for e in errs) <= MAX_ABS and max(e[1] for e in errs) <= MEAN_ABS
+
+
+def test_reference_growth_and_short_rows():
+    """Scores that keep growing along a row force the rescale of O on both softmax teams and
+    the merge of their sums; rows of one, two and three KV blocks exercise the hand-over of
+    the running reference at the start of a task."""
+    cfg = _small("wan480p", 3, 1)
+    w = Workload(cfg)
+    b, nb = cfg.block, cfg.n_blocks
+    # keys of block j scaled by 1 + 0.35 j: the row max rises by far more than 2^8 overall
+    k = w.k[0].float()
+    for j in range(nb):
+        k[j * b:(j + 1) * b] *= 1.0 + 0.35 * j
+    w.k[0].copy_(k.to(torch.bfloat16))
+    K64 = I.bf16_to_f64(w.k[0].cpu())
+    Q64, V64 = w.head_f64("q", 0), w.head_f64("v", 0)
+    # rows 0..2 get exactly 1, 2, 3 blocks; the others keep the generated lists
+    mask = w.masks[0].copy()
+    for r, cols in ((0, [0]), (1, [1, nb - 1]), (2, [0, 5, nb - 1])):
+        mask[r, :] = False
+        mask[r, cols] = True
+    w.masks[0] = mask
+    ptr_np, idx_np = I.masks_to_csr([mask])
+    w.ptr, w.idx = torch.from_numpy(ptr_np).cuda(), torch.from_numpy(idx_np).cuda()
+    lse = torch.empty((1, cfg.seq), dtype=torch.float32, device="cuda")
+    o, st = run_attention(w, lse=lse, scale=1.0)
+    assert st == [0, 0, 0, 0]
+    ref, ref_lse = wo.block_sparse_attention(Q64, K64, V64, mask, b, b, cfg.seq, cfg.seq, 1.0)
+    g = o[0, :cfg.seq].float().cpu().numpy()
+    assert np.isfinite(g).all()
+    mx, mean = error_stats(g, ref)
+    assert mx <= 4e-2 and mean <= MEAN_ABS, (mx, mean)      # near one-hot rows: bf16 rounding of O dominates
+    assert np.abs(lse[0].cpu().numpy() - ref_lse).max() < 5e-3 * max(1.0, np.abs(ref_lse).max() / 10)
