@@ -205,8 +205,8 @@ def run_waveal(args, cfg):
     if args.svd_iters > 0:
         pdesc.svd_iters = args.svd_iters
     pws = torch.empty((wb.plan_workspace_bytes(pdesc) + 256,), dtype=torch.uint8, device=dev)
-    aws = torch.empty((256,), dtype=torch.uint8, device=dev)
     adesc = wb.attn_desc(q, k, v, o, S, S, B, args.head_order == "interleaved")
+    aws = torch.empty((wb.bsattn_workspace_bytes(adesc),), dtype=torch.uint8, device=dev)
     status = torch.zeros((4,), dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
     launches = {"n": 0}

@@ -150,6 +150,14 @@ waveal_status waveal_bitmap_to_csr_noalloc(int32_t heads, int32_t n_q_blocks, in
 /* Largest heads * n_q_blocks the call above accepts.  Host-only. */
 size_t waveal_noalloc_max_rows(void);
 
+/* waveal_attn_desc.flags: take the row max of every KV block (the online-softmax rule as the
+ * paper's backends apply it) in a single launch.  Without the flag the kernel fixes each row's
+ * reference after the first two blocks of a task - softmax does not depend on the reference as
+ * long as nothing overflows - watches the size of every block's sum, lists the tasks where a
+ * sum reached 2^80 and computes those again, with the max of every block, in a second launch
+ * on the same stream.  Results agree to rounding; the flag exists for comparison runs. */
+#define WAVEAL_ATTN_ONLINE_MAX_ONLY 1
+
 typedef struct waveal_attn_desc {
   int32_t heads;            /* batch*heads; K/V heads == Q heads                              */
   int32_t seq_q, seq_kv;    /* true (unpadded) lengths                                        */
@@ -158,10 +166,12 @@ typedef struct waveal_attn_desc {
   int64_t q_stride[2], k_stride[2], v_stride[2], o_stride[2]; /* elements: {head, token}; head_dim contiguous */
   int32_t order_heads_interleaved; /* 0 = heads run one after another (Section 5, sequential
                                       heads); 1 = position-major across heads (parallel heads) */
-  int32_t reserved;
+  int32_t flags;            /* 0, or WAVEAL_ATTN_ONLINE_MAX_ONLY                               */
 } waveal_attn_desc;
 
-/* Bytes of device workspace waveal_bsattn_fwd needs (ticket counter + abort flag).  Host-only. */
+/* Bytes of device workspace waveal_bsattn_fwd needs: 32 bytes of counters (int32 words: ticket
+ * counter, abort flag, number of tasks computed twice, ticket counter of the second launch) and
+ * 8 bytes per (head, query block) for the list of tasks to compute again.  Host-only. */
 waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* desc /*host*/, size_t* bytes /*host*/);
 
 /* Block-sparse attention forward, bf16 in / fp32 accumulate / bf16 out (Sections 2.1-2.3):
@@ -175,7 +185,8 @@ waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* desc /*host*
  * lse: dev float [heads][seq_q] or NULL (natural-log sum-exp per query token; -inf for a
  * query block with an empty list, whose O is 0).
  * scale <= 0 means 1/sqrt(head_dim).
- * ws: dev workspace (waveal_bsattn_workspace_bytes), 16-byte aligned.
+ * ws: dev workspace (waveal_bsattn_workspace_bytes), 16-byte aligned; after the call its int32
+ * word 2 holds the number of tasks the second launch computed again (normally 0).
  * dev_status: dev int32 [4] or NULL: {code, site, block, aux}; written only on a device-side
  * failure (the caller zeroes it).
  * The first call in a process also looks up a driver entry point (no allocation). */

@@ -43,7 +43,7 @@ class AttnDesc(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("block_q", ctypes.c_int32), ("block_kv", ctypes.c_int32),
                 ("q_stride", ctypes.c_int64 * 2), ("k_stride", ctypes.c_int64 * 2), ("v_stride", ctypes.c_int64 * 2),
                 ("o_stride", ctypes.c_int64 * 2), ("order_heads_interleaved", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("flags", ctypes.c_int32)]
 
 
 class WavealError(RuntimeError):
@@ -245,7 +245,10 @@ def scatter_rows(src, dst, row_order, block: int, stream=None):
     _move_rows("waveal_scatter_rows", src, dst, row_order, block, stream)
 
 
-def attn_desc(q, k, v, o, seq_q: int, seq_kv: int, block: int, interleaved: bool = False) -> AttnDesc:
+ATTN_ONLINE_MAX_ONLY = 1
+
+
+def attn_desc(q, k, v, o, seq_q: int, seq_kv: int, block: int, interleaved: bool = False, flags: int = 0) -> AttnDesc:
     """Descriptor for [heads, tokens, head_dim] tensors (head_dim contiguous)."""
     d = AttnDesc()
     d.heads, d.seq_q, d.seq_kv, d.head_dim = q.shape[0], seq_q, seq_kv, q.shape[2]
@@ -254,6 +257,7 @@ def attn_desc(q, k, v, o, seq_q: int, seq_kv: int, block: int, interleaved: bool
         assert t.stride(2) == 1, "head_dim must be contiguous"
         getattr(d, name)[0], getattr(d, name)[1] = t.stride(0), t.stride(1)
     d.order_heads_interleaved = 1 if interleaved else 0
+    d.flags = flags
     return d
 
 

@@ -44,9 +44,9 @@ def measure(cfg, reps: int):
     pdesc = wb.plan_desc_default(heads=H, n_q_blocks=nb, n_kv_blocks=nb, wave_size=wb.default_wave_size(),
                                  mode=wb.FORCE_REORDER, seed=cfg.plan_seed, kv_bytes_per_head=2 * Sp * D * 2)
     pws = torch.empty((wb.plan_workspace_bytes(pdesc) + 256,), dtype=torch.uint8, device=dev)
-    aws = torch.empty((256,), dtype=torch.uint8, device=dev)
     st = torch.zeros((4,), dtype=torch.int32, device=dev)
     adesc = wb.attn_desc(q, k, v, o, S, S, B)
+    aws = torch.empty((wb.bsattn_workspace_bytes(adesc),), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
     def timed(fn):

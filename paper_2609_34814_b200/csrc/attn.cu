@@ -259,7 +259,9 @@ struct AttnParams {
   const int* row_ptr;
   const int* kv_idx;
   const int* row_order;
-  int* ws;            // [0] ticket counter, [1] abort flag
+  int* ws;            // [0] ticket counter, [1] abort flag, [2] number of tasks to redo, [3] ticket counter of
+                      // the redo pass, [8 + 2i], [9 + 2i] = (head, query block) of redo entry i
+  int redo_pass;      // 0: all tasks by ticket; 1: only the tasks the first pass listed
   int* dev_status;
   long long o_stride_h, o_stride_t;
   int heads, m_b, n_b, seq_q, seq_kv, interleaved;
@@ -296,7 +298,7 @@ struct Geo {
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
   static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
   static constexpr int OFF_MISC = OFF_MX + 2 * 128 * 4 + 2 * 2 * 128 * 8;
-  static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;   // + slack for 1024-byte alignment
+  static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;   // + slack for 1024-byte alignment
   // tensor memory: three S/P buffers of 128 columns, then the output accumulator
   static constexpr uint32_t S_STRIDE = 128, O_COL = 384, TMEM_COLS = 512;
 };
@@ -370,7 +372,7 @@ __device__ __forceinline__ bool warp_spin(const Ctx& c, uint32_t bar, uint32_t p
   return __all_sync(0xffffffffu, mbar_spin(c, bar, parity, site));
 }
 
-template <int BLOCK, int D>
+template <int BLOCK, int D, bool FAST>
 __global__ void __launch_bounds__(kThreads, 1)
 k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
              const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -380,6 +382,9 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // provably warp-uniform role index
+
+  // second pass with nothing listed (or after an abort): leave before anything is set up
+  if (p.redo_pass && (p.ws[2] == 0 || p.ws[1] != 0)) return;
 
   const uint32_t bar0 = sbase + G::OFF_BAR;
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -393,6 +398,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   float2* ex = reinterpret_cast<float2*>(smem + G::OFF_MX + 2 * 128 * 4);       // [task parity][team][128] (reference, sum)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + G::OFF_MISC);
   volatile int* abort_smem = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 4);
+  volatile int* redo_flag = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 8);   // [task parity]
   Ctx ctx{bar0, abort_smem, p.ws, p.dev_status};
 
   if (tid == 0) {
@@ -412,6 +418,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     mbar_init(BAR(B_FINAL), 1);
     for (int i = 0; i < 8; ++i) mbar_init(BAR(B_MX + i), 1);
     *abort_smem = 0;
+    redo_flag[0] = 0;
+    redo_flag[1] = 0;
     fence_mbar_init();
     fence_proxy_async();
   }
@@ -438,17 +446,26 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     uint32_t k_armed = 0, k_parity = 0, v_armed = 0, v_parity = 0;   // per stage: parity of the last load armed on it
     bool q_armed = false; uint32_t q_armed_parity = 0;
     while (ok) {
-      long long t = 0;
-      if (lane == 0) t = (p.ws[1] != 0) ? p.total_tasks : (long long)(unsigned)atomicAdd(&p.ws[0], 1);
+      long long t = 0, n_tasks = p.total_tasks;
+      if (lane == 0) {
+        if (p.redo_pass) n_tasks = min((long long)p.ws[2], p.total_tasks);   // written by the first pass
+        t = (p.ws[1] != 0) ? n_tasks : (long long)(unsigned)atomicAdd(&p.ws[p.redo_pass ? 3 : 0], 1);
+      }
       t = __shfl_sync(0xffffffffu, t, 0);
+      n_tasks = __shfl_sync(0xffffffffu, n_tasks, 0);
       Task tk{};
-      if (t >= p.total_tasks) {
+      if (t >= n_tasks) {
         tk.n = -1;
       } else {
-        int h, pos;
-        if (p.interleaved) { pos = (int)(t / p.heads); h = (int)(t % p.heads); }
-        else { h = (int)(t / p.m_b); pos = (int)(t % p.m_b); }
-        int row = p.row_order ? p.row_order[(size_t)h * p.m_b + pos] : pos;
+        int h, pos, row;
+        if (p.redo_pass) {
+          h = p.ws[8 + 2 * t]; row = p.ws[9 + 2 * t]; pos = row;
+          if (h < 0 || h >= p.heads) h = 0;
+        } else {
+          if (p.interleaved) { pos = (int)(t / p.heads); h = (int)(t % p.heads); }
+          else { h = (int)(t / p.m_b); pos = (int)(t % p.m_b); }
+          row = p.row_order ? p.row_order[(size_t)h * p.m_b + pos] : pos;
+        }
         if (row < 0 || row >= p.m_b) row = pos;          // never index out of range
         int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
         tk.h = h; tk.row = row; tk.lo = lo; tk.n = max(hi - lo, 0);
@@ -688,6 +705,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + slot));
       float2* exb = ex + (task_it & 1) * 256;
+      const uint32_t rslot = task_it & 1;
       ++task_it;
       if (tk.n < 0) break;
       const long long q_tok = (long long)tk.row * G::BQ + r;
@@ -715,7 +733,15 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #ifndef WAVEAL_DBG_NOSM   // (timing experiments only: with the macro the softmax warps just pass the barriers on)
           // ---- pass 1: row max (the values are loaded again for the exponentials: a second
           // tensor-memory load is cheaper than 128 live registers)
+          // In the first pass over the tasks (FAST) only blocks 0 and 1 of a task take a max and
+          // may move the reference; from block 2 on both teams keep the reference of block 1.
+          // Any reference gives the same softmax as long as nothing overflows, so the later
+          // blocks only watch the largest exponent they produce: if it ever exceeds 100 the
+          // task is put on a list and computed again by the second launch, which takes the
+          // max of every block (the rule of the paper's online softmax).
+          const bool fixed_ref = FAST && j >= 2;
           float mloc = -INFINITY;
+          if (!fixed_ref)
 #pragma unroll
           for (int ch = 0; ch < G::NCH; ++ch) {
             uint32_t sv[G::CH];
@@ -742,9 +768,9 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           }
           if (quad == 2) TRACE(1 + team, 12 + team, j);
           // ---- the row's reference after block j-1, from the other team
-          float m_prev = -INFINITY;
-          if (j > 0) {
-            // that team's arrival for block j-1 is phase number (blocks of that parity so far) - 1
+          float m_prev = m_ref;
+          if (j > 0 && (!fixed_ref || j == 2)) {
+            // that team's arrival for block j-1 is phase number (arrivals of that parity so far) - 1
             ok = warp_spin(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24);
             if (!ok) break;
             m_prev = mpub[(par ^ 1u) * 128 + r];
@@ -752,11 +778,13 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           const float m_cand = fmaxf(m_prev, mloc * p.sl2);
           // keep the stale reference unless it is exceeded by more than 2^8 (exact: the final
           // normalisation divides by a sum taken with the same reference)
-          const bool grow = __any_sync(0xffffffffu, m_cand > m_prev + 8.0f);
+          const bool grow = !fixed_ref && __any_sync(0xffffffffu, m_cand > m_prev + 8.0f);
           const float m_new = grow ? m_cand : m_prev;
-          mpub[par * 128 + r] = m_new;
-          __syncwarp();
-          if (lane == 0) mbar_arrive(BAR(B_MX + quad * 2 + par));
+          if (!fixed_ref) {
+            mpub[par * 128 + r] = m_new;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR(B_MX + quad * 2 + par));
+          }
           if (m_new != m_ref) {
             l_run *= (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
             m_ref = m_new;
@@ -798,7 +826,11 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             if constexpr (G::CH == 64) { WAVEAL_TMEM_ST32(s_addr + ch * 32, pk, 0); }
             else { WAVEAL_TMEM_ST16(s_addr + ch * 16, pk, 0); }
           }
-          l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+          const float l_blk = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+          l_run += l_blk;
+          // all terms are positive, so a block sum below 2^80 bounds every exponent of the block;
+          // above it (or not a number) the fixed reference is too far off: redo the task
+          if (fixed_ref && __any_sync(0xffffffffu, !(l_blk < 1.2089258e24f))) redo_flag[rslot] = 1;
           if (quad == 2) TRACE(1 + team, 14 + team, j);
           // rare: the reference grew, so O (blocks 0..j-1) is rescaled; its last MMA (block j-1)
           // must be complete: that is the latest phase of the barrier of the S buffer before
@@ -833,7 +865,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
         // both teams count every block
         s_phase ^= 1u << sb;
-        mx_phase ^= 1u << par;
+        if (!(FAST && j >= 2)) mx_phase ^= 1u << par;   // one flip per arrival on that parity's barrier
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
       if (!ok) break;
@@ -844,6 +876,14 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       ++o_it;
       tc_fence_after();
       if (quad == 2) TRACE(1 + team, 18 + team, tk.n);
+      if (FAST && sw == 0 && lane == 0 && redo_flag[rslot]) {
+        // every warp's blocks of this task lie before O_FULL; the slot is used again two tasks
+        // later, after this warp's O_FREE arrival below
+        const int e = atomicAdd(&p.ws[2], 1);
+        p.ws[8 + 2 * e] = tk.h;
+        p.ws[9 + 2 * e] = tk.row;
+        redo_flag[rslot] = 0;
+      }
       exb[team * 128 + r] = make_float2(m_ref, l_run);
       named_bar_sync(1 + quad, 64);
       const float2 oth = exb[(team ^ 1) * 128 + r];
@@ -948,12 +988,26 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   if ((s = make_map(&tq, Q, D, d->seq_q, d->heads, d->q_stride[0], d->q_stride[1], BLOCK, "Q")) != WAVEAL_OK) return s;
   if ((s = make_map(&tk, K, D, d->seq_kv, d->heads, d->k_stride[0], d->k_stride[1], BLOCK, "K")) != WAVEAL_OK) return s;
   if ((s = make_map(&tv, V, D, d->seq_kv, d->heads, d->v_stride[0], d->v_stride[1], BLOCK, "V")) != WAVEAL_OK) return s;
-  WAVEAL_CUDA_OK(cudaFuncSetAttribute(k_bsattn_fwd<BLOCK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES));
-  WAVEAL_CUDA_OK(cudaMemsetAsync(p.ws, 0, 16, st));  // ticket counter, abort flag (and the debug trace count)
+  WAVEAL_CUDA_OK(cudaFuncSetAttribute(k_bsattn_fwd<BLOCK, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES));
+  WAVEAL_CUDA_OK(cudaFuncSetAttribute(k_bsattn_fwd<BLOCK, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES));
+  WAVEAL_CUDA_OK(cudaMemsetAsync(p.ws, 0, 32, st));  // ticket counters, abort flag, redo count
   long long grid = p.total_tasks < sms ? p.total_tasks : sms;
-  k_bsattn_fwd<BLOCK, D><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
+  if (d->flags & WAVEAL_ATTN_ONLINE_MAX_ONLY) {
+    p.redo_pass = 0;
+    k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
+    WAVEAL_CUDA_OK(cudaGetLastError());
+    waveal::launch_counter() = 1;
+    return WAVEAL_OK;
+  }
+  // first pass: reference fixed after the first two blocks of a task; second pass: the tasks the
+  // first one listed (normally none: its CTAs leave at once), max of every block
+  p.redo_pass = 0;
+  k_bsattn_fwd<BLOCK, D, true><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
   WAVEAL_CUDA_OK(cudaGetLastError());
-  waveal::launch_counter() = 1;
+  p.redo_pass = 1;
+  k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
+  WAVEAL_CUDA_OK(cudaGetLastError());
+  waveal::launch_counter() = 2;
   return WAVEAL_OK;
 }
 
@@ -963,7 +1017,9 @@ extern "C" waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* d
   waveal_status s = check_desc(desc);
   if (s != WAVEAL_OK) return s;
   if (!bytes) return waveal::fail(WAVEAL_ERR_INVALID_ARG, "bytes is NULL");
-  *bytes = 256;
+  // 32 bytes of counters and flags, then one (head, query block) pair per task for the redo list
+  const long long m_b = (desc->seq_q + desc->block_q - 1) / desc->block_q;
+  *bytes = (size_t)(((32 + 8 * (long long)desc->heads * m_b) + 255) / 256 * 256);
   return WAVEAL_OK;
 }
 
@@ -977,7 +1033,9 @@ extern "C" waveal_status waveal_bsattn_fwd(const waveal_attn_desc* d, const void
   if (!kv_row_ptr || !kv_block_indices) return waveal::fail(WAVEAL_ERR_INVALID_ARG, "index lists are required");
   if (!waveal::aligned(Q, 16) || !waveal::aligned(K, 16) || !waveal::aligned(V, 16) || !waveal::aligned(O, 16))
     return waveal::fail(WAVEAL_ERR_INVALID_ARG, "Q, K, V and O must be 16-byte aligned");
-  if (!ws || ws_bytes < 256) return waveal::fail(WAVEAL_ERR_WORKSPACE, "workspace of 256 bytes needed");
+  size_t ws_need = 0;
+  if ((s = waveal_bsattn_workspace_bytes(d, &ws_need)) != WAVEAL_OK) return s;
+  if (!ws || ws_bytes < ws_need) return waveal::fail(WAVEAL_ERR_WORKSPACE, "workspace of %zu bytes needed", ws_need);
   if (!waveal::aligned(ws, 16)) return waveal::fail(WAVEAL_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
   if (!(scale == scale) || std::isinf(scale)) return waveal::fail(WAVEAL_ERR_INVALID_ARG, "scale is not finite");
   int dev = 0, sms = 0, major = 0;

@@ -209,3 +209,49 @@ def test_reference_growth_and_short_rows():
     mx, mean = error_stats(g, ref)
     assert mx <= 4e-2 and mean <= MEAN_ABS, (mx, mean)      # near one-hot rows: bf16 rounding of O dominates
     assert np.abs(lse[0].cpu().numpy() - ref_lse).max() < 5e-3 * max(1.0, np.abs(ref_lse).max() / 10)
+
+
+def test_second_launch_recomputes_tasks_whose_reference_was_too_low():
+    """Keys that are far larger in one late KV block push the exponents of the fixed-reference
+    pass over its limit: those tasks must be listed, computed again with the max of every
+    block, and agree with the oracle; harmless inputs list nothing."""
+    cfg = _small("wan480p", 3, 1)
+    w = Workload(cfg)
+    b, nb = cfg.block, cfg.n_blocks
+    d = wb.attn_desc(w.q, w.k, w.v, w.o, cfg.seq, cfg.seq, b)
+    ws = torch.zeros((wb.bsattn_workspace_bytes(d),), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    wb.bsattn_fwd(d, w.q, w.k, w.v, w.o, w.ptr, w.idx, workspace=ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.tolist() == [0, 0, 0, 0] and ws.view(torch.int32)[2].item() == 0
+    # block 20 of K scaled by 40: scores there exceed everything before them by far more than 2^100
+    jb = 20
+    k = w.k[0].float()
+    k[jb * b:(jb + 1) * b] *= 40.0
+    w.k[0].copy_(k.to(torch.bfloat16))
+    hit = [i for i in range(nb) if w.masks[0][i, jb] and np.nonzero(w.masks[0][i])[0].tolist().index(jb) >= 2]
+    assert len(hit) >= 3
+    o = torch.full_like(w.o, float("nan"))
+    ws.zero_()
+    wb.bsattn_fwd(d, w.q, w.k, w.v, o, w.ptr, w.idx, workspace=ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.tolist() == [0, 0, 0, 0]
+    n_redo = ws.view(torch.int32)[2].item()
+    listed = sorted(ws.view(torch.int32)[8:8 + 2 * n_redo].view(-1, 2)[:, 1].tolist())
+    assert n_redo >= 1 and set(listed) <= set(hit), (n_redo, listed, hit)
+    K64 = I.bf16_to_f64(w.k[0].cpu())
+    ref, _ = wo.block_sparse_attention(w.head_f64("q", 0), K64, w.head_f64("v", 0), w.masks[0], b, b, cfg.seq, cfg.seq)
+    g = o[0, :cfg.seq].float().cpu().numpy()
+    assert np.isfinite(g).all()
+    mx, mean = error_stats(g, ref)
+    assert mx <= 4e-2 and mean <= MEAN_ABS, (mx, mean)
+    # the single-launch variant that takes the max of every block gives the same rows for the listed tasks
+    o2 = torch.zeros_like(w.o)
+    d2 = wb.attn_desc(w.q, w.k, w.v, o2, cfg.seq, cfg.seq, b, flags=wb.ATTN_ONLINE_MAX_ONLY)
+    wb.bsattn_fwd(d2, w.q, w.k, w.v, o2, w.ptr, w.idx, workspace=ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert wb.last_launch_count() == 1
+    for i in listed:
+        assert torch.equal(o[0, i * b:min((i + 1) * b, cfg.seq)], o2[0, i * b:min((i + 1) * b, cfg.seq)])
+    mx2, mean2 = error_stats(o2[0, :cfg.seq].float().cpu().numpy(), ref)
+    assert mx2 <= 4e-2 and mean2 <= MEAN_ABS
