@@ -294,7 +294,7 @@ struct Geo {
   static constexpr int OFF_K = OFF_Q + Q_BYTES;
   static constexpr int OFF_V = OFF_K + NKS * TILE_BYTES;
   static constexpr int OFF_BAR = OFF_V + NVS * TILE_BYTES;
-  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 3 * NSBUF + 2 + 1 + 8;
+  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 4 * NSBUF + 2 + 1 + 8;
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
   static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
   static constexpr int OFF_MISC = OFF_MX + 2 * 128 * 4 + 2 * 2 * 128 * 8;
@@ -390,7 +390,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   constexpr int B_TASK_FULL = 0, B_TASK_EMPTY = 2, B_Q_FULL = 4, B_Q_EMPTY = 5, B_K_FULL = 6,
                 B_K_EMPTY = B_K_FULL + G::NKS, B_V_FULL = B_K_EMPTY + G::NKS, B_V_EMPTY = B_V_FULL + G::NVS,
-                B_S_FULL = B_V_EMPTY + G::NVS, B_P_FULL = B_S_FULL + G::NSBUF, B_S_FREE = B_P_FULL + G::NSBUF,
+                B_S_FULL = B_V_EMPTY + G::NVS, B_P_FULL = B_S_FULL + G::NSBUF, B_S_FREE = B_P_FULL + 2 * G::NSBUF,
                 B_O_FULL = B_S_FREE + G::NSBUF, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1, B_MX = B_FINAL + 1;
   static_assert(B_MX + 8 <= G::N_BAR, "barrier count");
   Task* tasks = reinterpret_cast<Task*>(smem + G::OFF_TASK);
@@ -410,7 +410,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     for (int i = 0; i < G::NVS; ++i) { mbar_init(BAR(B_V_FULL + i), 1); mbar_init(BAR(B_V_EMPTY + i), 1); }
     for (int i = 0; i < G::NSBUF; ++i) {
       mbar_init(BAR(B_S_FULL + i), 1);
-      mbar_init(BAR(B_P_FULL + i), 4);     // the four warps of the team that owns the block
+      mbar_init(BAR(B_P_FULL + 2 * i), 4);      // one per half of P (the four warps of the owning team)
+      mbar_init(BAR(B_P_FULL + 2 * i + 1), 4);
       mbar_init(BAR(B_S_FREE + i), 1);
     }
     mbar_init(BAR(B_O_FULL), 1);
@@ -631,35 +632,37 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (!ok) break;
       o_ph ^= 1;
       for (int j = 0; j < n && ok; ++j) {
-        ok = warp_spin(ctx, BAR(B_P_FULL + sb), (p_phase >> sb) & 1u, 14);
-        if (!ok) break;
-        p_phase ^= 1u << sb;
-        TRACE(0, 1, j);
-        ok = warp_spin(ctx, BAR(B_V_FULL + v_st), v_ph, 15);
-        if (!ok) break;
-        TRACE(0, 2, j);
-        tc_fence_after();
-        {
+        // P_j arrives in two halves (the first and the second half of the block's keys), each
+        // with its own barrier: the MMAs on the first half run while the softmax team is still
+        // computing the second
+        const uint64_t vd = vdesc0 + (uint64_t)(v_st * (uint32_t)(G::TILE_BYTES >> 4));
+        const uint32_t pbase = tmem_base + sb * G::S_STRIDE;
+        const uint32_t d_o = tmem_base + G::O_COL;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t pb = sb * 2 + h;
+          ok = warp_spin(ctx, BAR(B_P_FULL + pb), (p_phase >> pb) & 1u, 14);
+          if (!ok) break;
+          p_phase ^= 1u << pb;
+          if (h == 0) {
+            TRACE(0, 1, j);
+            ok = warp_spin(ctx, BAR(B_V_FULL + v_st), v_ph, 15);
+            if (!ok) break;
+            TRACE(0, 2, j);
+          }
+          tc_fence_after();
           // V tile as the N x K operand with N (head_dim) contiguous: 8 keys per 1024-byte
           // group along K (16 keys = 2048 bytes per MMA), next 64 columns of head_dim one slab further
-          const uint64_t vd = vdesc0 + (uint64_t)(v_st * (uint32_t)(G::TILE_BYTES >> 4));
-          const uint32_t pbase = tmem_base + sb * G::S_STRIDE;
-          const uint32_t d_o = tmem_base + G::O_COL;
-          if (j > 0) {
 #pragma unroll
-            for (int k = 0; k < G::BK / 16; ++k) {
+          for (int kk = 0; kk < G::BK / 32; ++kk) {
+            const int k = h * (G::BK / 32) + kk;
 #ifndef WAVEAL_DBG_SKIP_PV
-              umma_bf16_ts(d_o, pbase + k * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, 1u);
+            umma_bf16_ts(d_o, pbase + k * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
 #endif
-            }
-          } else {
-#pragma unroll
-            for (int k = 0; k < G::BK / 16; ++k) {
-#ifndef WAVEAL_DBG_SKIP_PV
-              umma_bf16_ts(d_o, pbase + k * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, k > 0 ? 1u : 0u);
-#endif
-            }
           }
+        }
+        if (!ok) break;
+        {
           tc_commit(BAR(B_V_EMPTY + v_st));
           tc_commit(BAR(B_S_FREE + sb));
           if (j == n - 1) tc_commit(BAR(B_O_FULL));
@@ -789,6 +792,26 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             l_run *= (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
             m_ref = m_new;
           }
+          // rare: the reference grew, so O (blocks 0..j-1) is rescaled; its last MMA (block j-1)
+          // must be complete: that is the latest phase of the barrier of the S buffer before
+          // this one (the next P V on that buffer needs a P this team has not produced yet).
+          // Done before any part of P_j is released to the MMA warp.
+          if (grow && j > 0) {
+            const uint32_t sbp = sb == 0 ? (uint32_t)G::NSBUF - 1u : sb - 1u;
+            ok = warp_wait(ctx, BAR(B_S_FREE + sbp), ((s_phase >> sbp) & 1u) ^ 1u, 22);
+            if (!ok) break;
+            tc_fence_after();
+            const float alpha = ex2(m_prev - m_new);
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+              uint32_t ov[32];
+              WAVEAL_TMEM_LD32(o_row + c0, ov, 0);
+              WAVEAL_TMEM_WAIT_LD32(ov, 0);
+#pragma unroll
+              for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
+              WAVEAL_TMEM_ST32(o_row + c0, ov, 0);
+            }
+          }
           // p' = 2^(s*scale*log2e - m + log2(1 + 2^-9)); P is p' cut to its top 16 bits (one byte
           // permute per pair instead of a conversion).  The extra factor centres the cut's error
           // around zero, like a rounding; the row sum adds the uncut p' and the epilogue takes
@@ -825,6 +848,13 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
             if constexpr (G::CH == 64) { WAVEAL_TMEM_ST32(s_addr + ch * 32, pk, 0); }
             else { WAVEAL_TMEM_ST16(s_addr + ch * 16, pk, 0); }
+            if (G::NCH == 2 && ch == 0) {
+              // first half of P_j: its MMAs can run while the second half is computed
+              tc_wait_st();
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb * 2));
+            }
           }
           const float l_blk = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
           l_run += l_blk;
@@ -832,25 +862,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           // above it (or not a number) the fixed reference is too far off: redo the task
           if (fixed_ref && __any_sync(0xffffffffu, !(l_blk < 1.2089258e24f))) redo_flag[rslot] = 1;
           if (quad == 2) TRACE(1 + team, 14 + team, j);
-          // rare: the reference grew, so O (blocks 0..j-1) is rescaled; its last MMA (block j-1)
-          // must be complete: that is the latest phase of the barrier of the S buffer before
-          // this one (the next P V on that buffer needs a P this team has not produced yet)
-          if (grow && j > 0) {
-            const uint32_t sbp = sb == 0 ? (uint32_t)G::NSBUF - 1u : sb - 1u;
-            ok = warp_wait(ctx, BAR(B_S_FREE + sbp), ((s_phase >> sbp) & 1u) ^ 1u, 22);
-            if (!ok) break;
-            tc_fence_after();
-            const float alpha = ex2(m_prev - m_new);
-#pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
-              uint32_t ov[32];
-              WAVEAL_TMEM_LD32(o_row + c0, ov, 0);
-              WAVEAL_TMEM_WAIT_LD32(ov, 0);
-#pragma unroll
-              for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-              WAVEAL_TMEM_ST32(o_row + c0, ov, 0);
-            }
-          }
 #else
           if (j > 0) { ok = warp_spin(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24); if (!ok) break; }
           __syncwarp();
@@ -860,7 +871,10 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           tc_wait_st();
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb));
+          if (lane == 0) {
+            if (G::NCH != 2) mbar_arrive(BAR(B_P_FULL + sb * 2));
+            mbar_arrive(BAR(B_P_FULL + sb * 2 + 1));
+          }
           if (quad == 2) TRACE(1 + team, 16 + team, j);
         }
         // both teams count every block
