@@ -25,6 +25,10 @@
 //               O in tensor memory is rescaled only when the max grew by more than 2^8; the
 //               epilogue adds the two sums, normalises and stores O at the ORIGINAL row (no
 //               inverse permutation)
+// Two launches per call: in the first the row max is taken in blocks 0 and 1 of a task only and
+// the reference stays fixed afterwards (softmax does not depend on it short of overflow); a task
+// in which a block's sum of exponentials reaches 2^80 is listed in the workspace and computed
+// again by the second launch, which takes the max of every block.
 // Every wait on an mbarrier is bounded; when one runs out the CTA records
 // {WAVEAL_ERR_TIMEOUT, site} and all roles leave through the common teardown.
 #include <cuda.h>
