@@ -84,18 +84,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-// non-blocking probe (try_wait may suspend the thread for a while when the phase is not complete)
-__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok;
-}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
@@ -358,24 +346,6 @@ __device__ __forceinline__ bool warp_wait(const Ctx& c, uint32_t bar, uint32_t p
   return __all_sync(0xffffffffu, mbar_wait(c, bar, parity, site));
 }
 
-// Latency-critical variant: polls with the non-suspending probe.  A suspended try_wait was
-// seen to resume several hundred cycles after the phase completed; a poll costs one issue
-// slot every few tens of cycles while it waits.
-__device__ __forceinline__ bool mbar_spin(const Ctx& c, uint32_t bar, uint32_t parity, int site) {
-  if (mbar_test_wait(bar, parity)) return true;
-  long long t0 = clock64();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_test_wait(bar, parity)) return true;
-    if (*c.abort_smem) return false;
-    if (clock64() - t0 > kTimeoutCycles) { signal_abort(c, site); return false; }
-  }
-}
-__device__ __forceinline__ bool warp_spin(const Ctx& c, uint32_t bar, uint32_t parity, int site) {
-  return __all_sync(0xffffffffu, mbar_spin(c, bar, parity, site));
-}
-
 template <int BLOCK, int D, bool FAST>
 __global__ void __launch_bounds__(kThreads, 1)
 k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -581,14 +551,14 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (!ok) break;
       q_ph ^= 1;
       for (int j = 0; j < n && ok; ++j) {
-        ok = warp_spin(ctx, BAR(B_K_FULL + k_st), k_ph, 12);
+        ok = warp_wait(ctx, BAR(B_K_FULL + k_st), k_ph, 12);
         if (!ok) break;
         // S[sb] also holds the P tile of the block that used it last: wait until that block's
         // P V has completed (its commit is phase number uses-1 of the buffer's barrier)
         if (first_uses > 0) {
           --first_uses;
         } else {
-          ok = warp_spin(ctx, BAR(B_S_FREE + sb), ((free_bits >> sb) & 1u) ^ 1u, 13);
+          ok = warp_wait(ctx, BAR(B_S_FREE + sb), ((free_bits >> sb) & 1u) ^ 1u, 13);
           if (!ok) break;
         }
         free_bits ^= 1u << sb;
@@ -645,12 +615,12 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const uint32_t pb = sb * 2 + h;
-          ok = warp_spin(ctx, BAR(B_P_FULL + pb), (p_phase >> pb) & 1u, 14);
+          ok = warp_wait(ctx, BAR(B_P_FULL + pb), (p_phase >> pb) & 1u, 14);
           if (!ok) break;
           p_phase ^= 1u << pb;
           if (h == 0) {
             TRACE(0, 1, j);
-            ok = warp_spin(ctx, BAR(B_V_FULL + v_st), v_ph, 15);
+            ok = warp_wait(ctx, BAR(B_V_FULL + v_st), v_ph, 15);
             if (!ok) break;
             TRACE(0, 2, j);
           }
@@ -731,7 +701,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       for (int j = 0; j < tk.n && ok; ++j) {
         const uint32_t par = (uint32_t)j & 1u;
         if ((int)par == team) {
-          ok = warp_spin(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
+          ok = warp_wait(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
           if (!ok) break;
           if (quad == 2) TRACE(1 + team, 10 + team, j);
           tc_fence_after();
@@ -778,7 +748,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           float m_prev = m_ref;
           if (j > 0 && (!fixed_ref || j == 2)) {
             // that team's arrival for block j-1 is phase number (arrivals of that parity so far) - 1
-            ok = warp_spin(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24);
+            ok = warp_wait(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24);
             if (!ok) break;
             m_prev = mpub[(par ^ 1u) * 128 + r];
           }
@@ -867,7 +837,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           if (fixed_ref && __any_sync(0xffffffffu, !(l_blk < 1.2089258e24f))) redo_flag[rslot] = 1;
           if (quad == 2) TRACE(1 + team, 14 + team, j);
 #else
-          if (j > 0) { ok = warp_spin(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24); if (!ok) break; }
+          if (j > 0) { ok = warp_wait(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24); if (!ok) break; }
           __syncwarp();
           if (lane == 0) mbar_arrive(BAR(B_MX + quad * 2 + par));
           l_run = 1.f; m_ref = 0.f;
