@@ -170,8 +170,9 @@ typedef struct waveal_attn_desc {
 } waveal_attn_desc;
 
 /* Bytes of device workspace waveal_bsattn_fwd needs: 32 bytes of counters (int32 words: ticket
- * counter, abort flag, number of tasks computed twice, ticket counter of the second launch) and
- * 8 bytes per (head, query block) for the list of tasks to compute again.  Host-only. */
+ * counter, abort flag, number of tasks computed twice, ticket counter of the second launch),
+ * 8 bytes per (head, query block) for the list of tasks to compute again and 32 bytes per
+ * (head, query block) for the table that maps a ticket to its task.  Host-only. */
 waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* desc /*host*/, size_t* bytes /*host*/);
 
 /* Block-sparse attention forward, bf16 in / fp32 accumulate / bf16 out (Sections 2.1-2.3):

@@ -245,6 +245,8 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 
 // ------------------------------------------------------------------ kernel
 
+struct Task { int h, row, lo, n, tail_valid, pad0, pad1, pad2; };
+
 struct AttnParams {
   __nv_bfloat16* O;
   float* lse;
@@ -254,6 +256,7 @@ struct AttnParams {
   int* ws;            // [0] ticket counter, [1] abort flag, [2] number of tasks to redo, [3] ticket counter of
                       // the redo pass, [8 + 2i], [9 + 2i] = (head, query block) of redo entry i
   int redo_pass;      // 0: all tasks by ticket; 1: only the tasks the first pass listed
+  const Task* table;         // task of every ticket of the first pass (k_task_table)
   int* dev_status;
   long long o_stride_h, o_stride_t;
   int heads, m_b, n_b, seq_q, seq_kv, interleaved;
@@ -261,7 +264,6 @@ struct AttnParams {
   float sl2;          // scale * log2(e)
 };
 
-struct Task { int h, row, lo, n, tail_valid, pad0, pad1, pad2; };
 
 template <int BLOCK, int D>
 struct Geo {
@@ -431,17 +433,15 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       Task tk{};
       if (t >= n_tasks) {
         tk.n = -1;
+      } else if (!p.redo_pass) {
+        // one 32-byte load behind the ticket instead of a chain through three lists
+        const uint4* e = reinterpret_cast<const uint4*>(p.table + t);
+        const uint4 a = e[0], b = e[1];
+        tk.h = (int)a.x; tk.row = (int)a.y; tk.lo = (int)a.z; tk.n = (int)a.w; tk.tail_valid = (int)b.x;
       } else {
-        int h, pos, row;
-        if (p.redo_pass) {
-          h = p.ws[8 + 2 * t]; row = p.ws[9 + 2 * t]; pos = row;
-          if (h < 0 || h >= p.heads) h = 0;
-        } else {
-          if (p.interleaved) { pos = (int)(t / p.heads); h = (int)(t % p.heads); }
-          else { h = (int)(t / p.m_b); pos = (int)(t % p.m_b); }
-          row = p.row_order ? p.row_order[(size_t)h * p.m_b + pos] : pos;
-        }
-        if (row < 0 || row >= p.m_b) row = pos;          // never index out of range
+        int h = p.ws[8 + 2 * t], row = p.ws[9 + 2 * t];
+        if (h < 0 || h >= p.heads) h = 0;
+        if (row < 0 || row >= p.m_b) row = 0;
         int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
         tk.h = h; tk.row = row; tk.lo = lo; tk.n = max(hi - lo, 0);
         tk.tail_valid = G::BK;
@@ -915,6 +915,25 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   }
 }
 
+// Task of every ticket (head-major or position-major over the planned order), so that the
+// persistent CTAs need one load behind a ticket instead of a chain through row_order, the row
+// pointers and the index list.
+__global__ void k_task_table(AttnParams p, int block_k, Task* table) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= p.total_tasks) return;
+  int h, pos;
+  if (p.interleaved) { pos = (int)(t / p.heads); h = (int)(t % p.heads); }
+  else { h = (int)(t / p.m_b); pos = (int)(t % p.m_b); }
+  int row = p.row_order ? p.row_order[(size_t)h * p.m_b + pos] : pos;
+  if (row < 0 || row >= p.m_b) row = pos;          // never index out of range
+  const int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
+  Task tk{};
+  tk.h = h; tk.row = row; tk.lo = lo; tk.n = max(hi - lo, 0);
+  tk.tail_valid = block_k;
+  if (tk.n > 0 && (p.seq_kv % block_k) != 0 && p.kv_idx[hi - 1] == p.n_b - 1) tk.tail_valid = p.seq_kv % block_k;
+  table[t] = tk;
+}
+
 // ------------------------------------------------------------------ host side
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -967,6 +986,9 @@ waveal_status check_desc(const waveal_attn_desc* d) {
   return WAVEAL_OK;
 }
 
+// byte offset of the ticket table in the workspace (32-byte aligned, behind header and redo list)
+long long table_offset(long long tasks) { return (32 + 8 * tasks + 31) / 32 * 32; }
+
 template <int BLOCK, int D>
 waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, const void* V, AttnParams& p,
                      int sms, cudaStream_t st) {
@@ -980,11 +1002,16 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   WAVEAL_CUDA_OK(cudaFuncSetAttribute(k_bsattn_fwd<BLOCK, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES));
   WAVEAL_CUDA_OK(cudaMemsetAsync(p.ws, 0, 32, st));  // ticket counters, abort flag, redo count
   long long grid = p.total_tasks < sms ? p.total_tasks : sms;
+  Task* table = reinterpret_cast<Task*>(reinterpret_cast<char*>(p.ws) + table_offset(p.total_tasks));
+  p.table = table;
+  p.redo_pass = 0;
+  k_task_table<<<(unsigned)((p.total_tasks + 255) / 256), 256, 0, st>>>(p, BLOCK, table);
+  WAVEAL_CUDA_OK(cudaGetLastError());
   if (d->flags & WAVEAL_ATTN_ONLINE_MAX_ONLY) {
     p.redo_pass = 0;
     k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
     WAVEAL_CUDA_OK(cudaGetLastError());
-    waveal::launch_counter() = 1;
+    waveal::launch_counter() = 2;
     return WAVEAL_OK;
   }
   // first pass: reference fixed after the first two blocks of a task; second pass: the tasks the
@@ -995,7 +1022,7 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   p.redo_pass = 1;
   k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
   WAVEAL_CUDA_OK(cudaGetLastError());
-  waveal::launch_counter() = 2;
+  waveal::launch_counter() = 3;
   return WAVEAL_OK;
 }
 
@@ -1005,9 +1032,10 @@ extern "C" waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* d
   waveal_status s = check_desc(desc);
   if (s != WAVEAL_OK) return s;
   if (!bytes) return waveal::fail(WAVEAL_ERR_INVALID_ARG, "bytes is NULL");
-  // 32 bytes of counters and flags, then one (head, query block) pair per task for the redo list
-  const long long m_b = (desc->seq_q + desc->block_q - 1) / desc->block_q;
-  *bytes = (size_t)(((32 + 8 * (long long)desc->heads * m_b) + 255) / 256 * 256);
+  // 32 bytes of counters and flags, one (head, query block) pair per task for the redo list,
+  // then the 32-byte task of every ticket
+  const long long tasks = (long long)desc->heads * ((desc->seq_q + desc->block_q - 1) / desc->block_q);
+  *bytes = (size_t)((table_offset(tasks) + 32 * tasks + 255) / 256 * 256);
   return WAVEAL_OK;
 }
 

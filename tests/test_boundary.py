@@ -75,10 +75,11 @@ def test_attention_host_errors_before_any_launch(lib):
         s[0], s[1] = 256 * 128, 128
     n = ctypes.c_size_t()
     assert lib.waveal_bsattn_workspace_bytes(ctypes.byref(d), ctypes.byref(n)) == wb.OK
-    assert n.value == 256                                # 32 bytes of counters + 8 per (head, query block), in units of 256
+    assert n.value == 256                                # counters + 8 + 32 bytes per (head, query block), in units of 256
     d.heads, d.seq_q = 40, 75600
     assert lib.waveal_bsattn_workspace_bytes(ctypes.byref(d), ctypes.byref(n)) == wb.OK
-    assert n.value == (32 + 8 * 40 * 591 + 255) // 256 * 256
+    tasks = 40 * 591
+    assert n.value == ((32 + 8 * tasks + 31) // 32 * 32 + 32 * tasks + 255) // 256 * 256
     d.heads, d.seq_q = 2, 256
     call = lambda q=0x1000, ws=0x9000, wsb=256, scale=0.0: lib.waveal_bsattn_fwd(
         ctypes.byref(d), q, 0x2000, 0x3000, 0x4000, None, 0x5000, 0x6000, None, ctypes.c_float(scale), ws, wsb,

@@ -250,7 +250,7 @@ def test_second_launch_recomputes_tasks_whose_reference_was_too_low():
     d2 = wb.attn_desc(w.q, w.k, w.v, o2, cfg.seq, cfg.seq, b, flags=wb.ATTN_ONLINE_MAX_ONLY)
     wb.bsattn_fwd(d2, w.q, w.k, w.v, o2, w.ptr, w.idx, workspace=ws, dev_status=st)
     torch.cuda.synchronize()
-    assert wb.last_launch_count() == 1
+    assert wb.last_launch_count() == 2               # ticket table + one attention launch
     for i in listed:
         assert torch.equal(o[0, i * b:min((i + 1) * b, cfg.seq)], o2[0, i * b:min((i + 1) * b, cfg.seq)])
     mx2, mean2 = error_stats(o2[0, :cfg.seq].float().cpu().numpy(), ref)
