@@ -343,7 +343,9 @@ __device__ __forceinline__ bool mbar_wait(const Ctx& c, uint32_t bar, uint32_t p
   }
 }
 
-// same, with one answer for the whole warp (the roles use warp-collective instructions)
+// same, with one answer for the whole warp (the roles use warp-collective instructions).  All
+// lanes wait: a warp suspended as a whole in try_wait takes no issue slots, which measured
+// better than polling and far better than one waiting lane with the rest at the vote.
 __device__ __forceinline__ bool warp_wait(const Ctx& c, uint32_t bar, uint32_t parity, int site) {
   return __all_sync(0xffffffffu, mbar_wait(c, bar, parity, site));
 }
