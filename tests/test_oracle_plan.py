@@ -215,6 +215,90 @@ def test_start_block_is_counter_based_and_in_range():
     assert wo._splitmix64(0) == 0xE220A8397B1DCDAF
 
 
+# the first three outputs of the published splitmix64 generator started from state 0 (the
+# generator adds the golden-ratio constant to its state before every mix, so output n is the
+# mix of n * golden)
+SPLITMIX_SEED0 = (0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F)
+GOLDEN64 = 0x9E3779B97F4A7C15
+
+
+def _unit(z):
+    """2u - 1 with u the top 53 bits of z as a fraction of 2^53, in exact integer arithmetic."""
+    from fractions import Fraction
+    return float(2 * Fraction(z >> 11, 1 << 53) - 1)
+
+
+def test_start_block_known_answers_fix_the_index_mixing():
+    o1, o2, o3 = SPLITMIX_SEED0
+    assert wo._splitmix64(GOLDEN64) == o2 and wo._splitmix64((2 * GOLDEN64) & (2 ** 64 - 1)) == o3
+    # seed 0, head 0: entry (0, 0) mixes counter 0
+    x = wo.start_block(0, 0, 4)
+    assert x[0, 0] == _unit(o1)
+    # the head enters as head * golden: head 1 / head 2 at counter 0 are outputs two and three
+    assert wo.start_block(0, 1, 4)[0, 0] == _unit(o2)
+    assert wo.start_block(0, 2, 4)[0, 0] == _unit(o3)
+    # the seed is xor-ed in: seed = golden cancels head 1, seed = golden at head 0 is output two
+    assert wo.start_block(GOLDEN64, 1, 4)[0, 0] == _unit(o1)
+    assert wo.start_block(GOLDEN64, 0, 4)[0, 0] == _unit(o2)
+    # the counter of entry (i, k) is 2i + k: seed 5 cancels it at (2, 1) only, seed 6 at (3, 0) only
+    x5 = wo.start_block(5, 0, 4)
+    assert x5[2, 1] == _unit(o1) and (x5 == _unit(o1)).sum() == 1
+    x6 = wo.start_block(6, 0, 4)
+    assert x6[3, 0] == _unit(o1) and (x6 == _unit(o1)).sum() == 1
+    x5h = wo.start_block(5, 1, 4)
+    assert x5h[2, 1] == _unit(o2) and (x5h == _unit(o2)).sum() == 1
+    # value map: o1 has its top bit set, o3 does not, so the signs differ
+    assert 0.76 < _unit(o1) < 0.77 and _unit(o3) < -0.94
+
+
+def test_fix_sign_is_flip_invariant_and_picks_the_first_large_entry():
+    rng = np.random.default_rng(0)
+    for _ in range(20):
+        u = rng.standard_normal(17)
+        a, b = wo.fix_sign(u), wo.fix_sign(-u)
+        assert np.array_equal(a, b)
+        assert np.array_equal(np.abs(a), np.abs(u))
+        i = int(np.nonzero(np.abs(u) >= 0.5 * np.abs(u).max())[0][0])
+        assert a[i] > 0
+    # symmetric +- ties of the largest magnitude: the first qualifying entry decides, not the maximum
+    u = np.array([0.1, -0.6, 1.0, -1.0, 0.6])
+    assert wo.fix_sign(u).tolist() == [-0.1, 0.6, -1.0, 1.0, -0.6]
+    assert wo.fix_sign(-u).tolist() == [-0.1, 0.6, -1.0, 1.0, -0.6]
+    # an entry just below half of the maximum does not qualify
+    u = np.array([-0.49, 1.0, -1.0])
+    assert wo.fix_sign(u).tolist() == [-0.49, 1.0, -1.0]
+    u = np.array([-0.5, 1.0, -1.0])
+    assert wo.fix_sign(u).tolist() == [0.5, -1.0, 1.0]
+    assert wo.fix_sign(np.zeros(4)).tolist() == [0, 0, 0, 0]
+
+
+def test_plan_head_ablation_modes_are_the_single_stages():
+    cfg = I.CONFIGS["wan480p"]
+    mk = I.make_mask(cfg, 2)
+    W = 37
+    ident = np.arange(cfg.n_blocks)
+    s1 = wo.plan_head(mk, W, 5, 9, 2, mode=wo.MODE_STAGE1_ONLY)
+    both = wo.plan_head(mk, W, 5, 9, 2, mode=wo.MODE_FORCE_REORDER)
+    s2 = wo.plan_head(mk, W, 5, 9, 2, mode=wo.MODE_STAGE2_ONLY)
+    nat = wo.plan_head(mk, W, 5, 9, 2, mode=wo.MODE_FORCE_NATURAL)
+    # Stage 1 alone: the angular order, untouched by the per-wave sort, and the same one S1+S2 starts from
+    assert np.array_equal(s1["row_order"], s1["order1"])
+    assert np.array_equal(s1["order1"], both["order1"])
+    assert np.array_equal(s1["order1"], wo.stage1_order(wo.polar_angles(s1["u"])))
+    assert not np.array_equal(s1["row_order"], ident)
+    # Stage 2 alone: natural order cut into waves, each sorted by descending count (no embedding)
+    assert np.array_equal(s2["order1"], ident)
+    assert np.array_equal(s2["row_order"], wo.stage2_order(ident, wo.row_nnz(mk), W))
+    exp = []
+    for lo in range(0, cfg.n_blocks, W):
+        exp += sorted(range(lo, min(lo + W, cfg.n_blocks)), key=lambda r: -int(mk[r].sum()))
+    assert s2["row_order"].tolist() == exp
+    assert np.abs(s2["u"]).max() == 0
+    # S1+S2 = Stage 2 applied to Stage 1's order
+    assert np.array_equal(both["row_order"], wo.stage2_order(s1["order1"], wo.row_nnz(mk), W))
+    assert np.array_equal(nat["row_order"], ident) and nat["flags"] & wo.FLAG_SKIPPED
+
+
 def test_plan_is_valid_permutation_and_bucket_invariants():
     cfg = I.CONFIGS["wan480p"]
     mk = I.make_mask(cfg, 1)
