@@ -7,9 +7,10 @@ the planned row order, over one synthetic video-shaped batch.
     python bench.py --impl reference ...                      # the CPU oracle, bounded sample
 
 Prints ONE JSON line (rank 0).  metric: TFLOP/s over computed block pairs
-(4 * block_q * block_kv * head_dim * #pairs / time).  With N > 1 every rank runs one batch
-element of the same shape (heads sharded by batch element, no data-path collective), timing
-is the max over ranks and the value is the whole-job aggregate ("weak" scaling).
+(4 * block_q * block_kv * head_dim * #pairs / time).  With N > 1 the heads of the one batch
+element are split over the ranks (contiguous slices, no data-path collective: heads are planned
+and attended independently), timing is the max over ranks and the value is all heads' FLOPs over
+that time ("strong" scaling); --replicas gives every rank a whole batch element instead ("weak").
 """
 from __future__ import annotations
 
@@ -18,9 +19,7 @@ import json
 import math
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 import numpy as np
@@ -41,55 +40,21 @@ def peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
-def ncu_traffic(workload: str):
-    """DRAM bytes per launch of the attention kernel from the committed ncu summary, if any."""
+def ncu_counters(workload: str):
+    """Counters of one launch of the attention kernel on this workload, per row order, from the
+    committed ncu summary (profiles/k_bsattn_fwd_<workload>.txt, lines `key: value`), if any."""
     p = os.path.join(ROOT, "profiles", f"k_bsattn_fwd_{workload}.txt")
+    out = {}
     if os.path.exists(p):
         for line in open(p):
-            if line.startswith("dram_bytes_per_launch_bench_workload:"):
-                return float(line.split(":")[1].split()[0])
-    return None
-
-
-class ClockSampler:
-    """nvidia-smi clock/throttle samples during the timed region (reading only)."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
-
-    def __init__(self, index: int):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.p = None
-        try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "20", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
-        except OSError:
-            pass
-
-    def stop(self):
-        if self.p is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.p.kill()
-        self.f.flush()
-        rows = [r.strip().split(", ") for r in open(self.f.name) if r.strip()]
-        os.unlink(self.f.name)
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-            except (ValueError, IndexError):
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.strip().lower().startswith("active"):
-                    reasons.add(n)
-        busy = sorted(sm)[len(sm) // 2:] if sm else []
-        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+            k, _, v = line.partition(":")
+            if k in ("l2_hit_pct_reordered", "l2_hit_pct_natural", "dram_read_bytes_reordered",
+                     "dram_write_bytes_reordered", "dram_read_bytes_natural", "dram_write_bytes_natural"):
+                try:
+                    out[k] = float(v.split()[0])
+                except (ValueError, IndexError):
+                    pass
+    return out
 
 
 # --------------------------------------------------------------------------- oracle legs
@@ -165,6 +130,7 @@ def run_waveal(args, cfg):
     from paper_2609_34814_b200 import binding as wb
     from paper_2609_34814_b200 import dist as wd
     from paper_2609_34814_b200 import inputs as I
+    from paper_2609_34814_b200 import timing as wt
 
     rank, world, local = wd.init("nccl")
     if not torch.cuda.is_available():
@@ -172,25 +138,31 @@ def run_waveal(args, cfg):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     wb.load()
-    H, S, Sp, D, B = cfg.heads, cfg.seq, cfg.seq_pad, cfg.head_dim, cfg.block
+    S, Sp, D, B = cfg.seq, cfg.seq_pad, cfg.head_dim, cfg.block
     nb = cfg.n_blocks
-    # ---- synthetic batch element of this rank: host (pinned) and device copies
+    # ---- this rank's heads: all of them at N = 1 or with --replicas, else a contiguous slice
+    split = world > 1 and not args.replicas
+    my_heads = list(wd.head_slice(rank, world, cfg.heads)) if split else list(range(cfg.heads))
+    H = len(my_heads)
+    if H == 0:
+        raise RuntimeError(f"{cfg.heads} heads cannot be split over {world} ranks")
+    # ---- synthetic inputs of those heads: host (pinned) and device copies
     if args.mask == "random20":
         # the unstructured mask of the paper's Table 1 (20 % uniform columns per row): the locality floor
-        masks = [I.random_mask(nb, nb, 0.20, cfg.mask_seed * 1000 + h) for h in range(H)]
+        masks = [I.random_mask(nb, nb, 0.20, cfg.mask_seed * 1000 + h) for h in my_heads]
     elif args.mask == "dense":
         # all block pairs: the dense run behind the gap metric (1/density) / (t_dense / t_sparse)
-        masks = [np.ones((nb, nb), dtype=bool) for _ in range(H)]
+        masks = [np.ones((nb, nb), dtype=bool) for _ in my_heads]
     else:
-        masks = [I.make_mask(cfg, h) for h in range(H)]
+        masks = [I.make_mask(cfg, h) for h in my_heads]
     bitmap_h = torch.from_numpy(np.stack([I.mask_to_bitmap(m) for m in masks]).view(np.int64)).pin_memory()
     ptr_np, idx_np = I.masks_to_csr(masks)
     pairs = int(ptr_np[-1])
-    flops = 4.0 * B * B * D * pairs
+    flops = 4.0 * B * B * D * pairs                         # this rank's share
     qkv_h = [torch.empty((H, Sp, D), dtype=torch.bfloat16).pin_memory() for _ in range(3)]
-    for h in range(H):
+    for i, h in enumerate(my_heads):
         for t, name in zip(qkv_h, "qkv"):
-            t[h].copy_(I.make_head_tensor(cfg, name, h))
+            t[i].copy_(I.make_head_tensor(cfg, name, h))
     o_h = torch.empty((H, Sp, D), dtype=torch.bfloat16).pin_memory()
     q, k, v = (t.to(dev, non_blocking=True) for t in qkv_h)
     o = torch.zeros_like(q)
@@ -207,58 +179,62 @@ def run_waveal(args, cfg):
     pws = torch.empty((wb.plan_workspace_bytes(pdesc) + 256,), dtype=torch.uint8, device=dev)
     adesc = wb.attn_desc(q, k, v, o, S, S, B, args.head_order == "interleaved")
     aws = torch.empty((wb.bsattn_workspace_bytes(adesc),), dtype=torch.uint8, device=dev)
+    aws_words = aws.view(torch.int32)
     status = torch.zeros((4,), dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
     launches = {"n": 0}
 
-    def step(mode=step_mode, count=False):
-        pdesc.mode = mode
+    def attend(order):
+        wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=order, workspace=aws, dev_status=status, stream=stream)
+
+    def step():
         plan = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream)
-        if count:
-            launches["n"] += wb.last_launch_count()
-        wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=plan.row_order, workspace=aws, dev_status=status,
-                      stream=stream)
-        if count:
-            launches["n"] += wb.last_launch_count()
+        attend(plan.row_order)
         return plan
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
+
+    def check_status():
+        if status.tolist()[0] != 0:
+            raise RuntimeError(f"device-side failure reported by the attention kernel: {status.tolist()}")
 
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
     # ---- timed region: K steps, events on the launching stream; the attention kernel of each
     #      step is bracketed by its own events for the roofline figure
-    pdesc.mode = step_mode
     attn_ev = []
+    cyc_log = torch.zeros((args.steps,), dtype=torch.int32, device=dev)
     wd.barrier()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local) if rank == 0 else None
+    sampler = wt.ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.begin("timed steps")
     e0, e1 = ev(), ev()
     e0.record(stream)
-    for _ in range(args.steps):
+    for i in range(args.steps):
         plan = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream)
         launches["n"] += wb.last_launch_count()
         a0, a1 = ev(), ev()
         a0.record(stream)
-        wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=plan.row_order, workspace=aws, dev_status=status,
-                      stream=stream)
+        attend(plan.row_order)
         a1.record(stream)
         launches["n"] += wb.last_launch_count()
         attn_ev.append((a0, a1))
     e1.record(stream)
     torch.cuda.synchronize()
+    if sampler:
+        sampler.end("timed steps")
     wd.barrier()
-    clocks = sampler.stop() if sampler else None
     total_ms = wd.max_over_ranks(e0.elapsed_time(e1), dev)
     ms_per_step = total_ms / args.steps
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_ev)
-    if status.tolist()[0] != 0:
-        raise RuntimeError(f"device-side failure reported by the attention kernel: {status.tolist()}")
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    check_status()
+    flops_all = wd.sum_over_ranks(flops, dev) if world > 1 else flops
+    value = flops_all / (ms_per_step * 1e-3) / 1e12
 
-    # ---- context numbers (outside the timed region): natural order, guard decision, plan alone
+    # ---- context numbers (outside the timed region)
     def timed(fn, reps=5):
         ts = []
         for _ in range(reps):
@@ -268,10 +244,19 @@ def run_waveal(args, cfg):
             ts.append(a.elapsed_time(b))
         return statistics.median(ts)
 
+    # planned vs natural row order of the same kernel: interleaved launches, per-pair ratios,
+    # and the kernel's own cycle counts (clock-independent)
     pdesc.mode = wb.FORCE_REORDER
     reo = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream).row_order
-    t_reo = timed(lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=reo, workspace=aws, dev_status=status, stream=stream))
-    t_nat = timed(lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=None, workspace=aws, dev_status=status, stream=stream))
+    if sampler:
+        torch.cuda.synchronize()
+        sampler.begin("order comparison")
+    ab = wt.ab_interleaved(lambda: attend(reo), lambda: attend(None), args.ab_pairs, stream,
+                           cycles_of=lambda: aws_words[4:5])
+    if sampler:
+        sampler.end("order comparison")
+    check_status()
+    t_reo, t_nat = ab["a_ms"], ab["b_ms"]
     t_plan = timed(lambda: wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream))
     pdesc.mode = wb.AUTO
     auto = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream)
@@ -343,39 +328,72 @@ def run_waveal(args, cfg):
         b.record(stream)
         torch.cuda.synchronize()
         wd.barrier()
-        if status.tolist()[0] != 0:
-            raise RuntimeError(f"device-side failure reported by the attention kernel: {status.tolist()}")
+        check_status()
         ms = wd.max_over_ranks(a.elapsed_time(b), dev) / n_e2e
         h2d = sum(t.numel() * t.element_size() for t in qkv_h) + bitmap_h.numel() * 8
-        e2e = {"value": world * flops / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
+        e2e = {"value": flops_all / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": o_h.numel() * 2,
                "pipeline": "%d groups of %d heads on three streams" % (len(groups), G)}
+
+    # ---- optional: every rank gets the whole O back (one all-gather over the head axis)
+    gather_ms = None
+    if split and args.gather_o:
+        torch.cuda.synchronize()
+        wd.barrier()
+        a, b = ev(), ev()
+        a.record(stream)
+        full = wd.gather_heads(o, cfg.heads)
+        b.record(stream)
+        torch.cuda.synchronize()
+        gather_ms = wd.max_over_ranks(a.elapsed_time(b), dev)
+        assert full.shape[0] == cfg.heads
+        del full
 
     pk = peaks()
     if rank != 0:
         wd.shutdown()
         return
     achieved = flops / (attn_ms * 1e-3) / 1e12
+    ctr = ncu_counters(cfg.name) if args.mask == "videomask" and not split else {}
+    traffic = None
+    key = "natural" if args.plan_mode == "natural" else "reordered"
+    if f"dram_read_bytes_{key}" in ctr and f"dram_write_bytes_{key}" in ctr:
+        traffic = ctr[f"dram_read_bytes_{key}"] + ctr[f"dram_write_bytes_{key}"]
+    clocks = sampler.summary("timed steps")
+    clocks_ab = sampler.summary("order comparison")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "heads": H, "head_dim": D, "seq": S, "block": B, "block_pairs": pairs,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if split else "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "heads": cfg.heads, "heads_per_rank": H, "head_dim": D, "seq": S, "block": B,
+                   "block_pairs_rank0": pairs,
                    "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode,
                    "mask": args.mask, "head_order": args.head_order, "svd_iters": int(pdesc.svd_iters),
-                   "step": "plan + attention", "l2": "inputs (Q,K,V,O %.1f GB) larger than L2, no flush" %
-                   (4 * H * Sp * D * 2 / 1e9), "batch_elements": world},
+                   "step": "plan + attention", "l2": "inputs (Q,K,V,O %.1f GB per rank) larger than L2, no flush" %
+                   (4 * H * Sp * D * 2 / 1e9),
+                   "sharding": ("heads split over ranks, no collective" if split else
+                                "one batch element per rank" if world > 1 else "single GPU")},
         "roofline": {"bound": "tensor", "kernel": "k_bsattn_fwd", "achieved": achieved, "peak": pk["bf16"],
                      "unit": "TFLOP/s", "frac": achieved / pk["bf16"], "peak_source": pk["source"] + " (burst)",
                      "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
-                     "kernel_ms": attn_ms,
-                     "traffic": ncu_traffic(cfg.name) if args.mask == "videomask" else None},
-        "kernel": {"attn_ms_reordered": t_reo, "attn_ms_natural": t_nat, "speedup_vs_natural": t_nat / t_reo,
+                     "kernel_ms": attn_ms, "traffic": traffic,
+                     "traffic_source": "ncu, one launch of this workload (profiles/)" if traffic else None},
+        "counters": {"source": "profiles/k_bsattn_fwd_%s.txt (ncu, one launch per order)" % cfg.name, **ctr} if ctr else None,
+        "kernel": {"attn_ms_reordered": t_reo, "attn_ms_natural": t_nat,
+                   "speedup_vs_natural": ab["b_over_a"], "speedup_vs_natural_min": ab["b_over_a_min"],
+                   "speedup_vs_natural_max": ab["b_over_a_max"],
+                   "speedup_vs_natural_cycles": ab.get("b_over_a_cycles"),
+                   "speedup_vs_natural_cycles_min": ab.get("b_over_a_cycles_min"),
+                   "speedup_vs_natural_cycles_max": ab.get("b_over_a_cycles_max"),
+                   "cycles_reordered": ab.get("a_cycles"), "cycles_natural": ab.get("b_cycles"),
+                   "comparison": "%d interleaved pairs, median of per-pair ratios" % ab["pairs"],
+                   "clocks_during_comparison": clocks_ab,
                    "tflops_reordered": flops / t_reo / 1e9, "tflops_natural": flops / t_nat / 1e9,
                    "plan_ms": t_plan, "plan_ms_auto": t_plan_auto, "auto_skipped_heads": skipped,
                    "plan_share_of_step": t_plan / (t_plan + t_reo),
                    "paper_gather_q_ms": t_gather, "paper_scatter_o_ms": t_scatter,
-                   "gather_gbs": copy_bytes / t_gather / 1e6, "gather_frac_of_hbm_peak": copy_bytes / t_gather / 1e6 / pk["hbm"]},
+                   "gather_gbs": copy_bytes / t_gather / 1e6, "gather_frac_of_hbm_peak": copy_bytes / t_gather / 1e6 / pk["hbm"],
+                   "all_gather_o_ms": gather_ms},
         "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
     }
     if world == 1 and not args.no_cpu:
@@ -404,6 +422,10 @@ def main():
     ap.add_argument("--head-order", default="sequential", choices=["sequential", "interleaved"],
                     help="ticket order: all rows of a head before the next head, or position-major over heads")
     ap.add_argument("--svd-iters", type=int, default=0, help="T of Algorithm 1 (0 = the library default)")
+    ap.add_argument("--ab-pairs", type=int, default=12, help="interleaved launch pairs of the planned-vs-natural comparison")
+    ap.add_argument("--replicas", action="store_true", help="N > 1: every rank runs a whole batch element (weak scaling) "
+                                                             "instead of a slice of the heads")
+    ap.add_argument("--gather-o", action="store_true", help="N > 1: also time the all-gather that re-assembles O on every rank")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

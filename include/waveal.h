@@ -25,6 +25,15 @@
  *     [heads*n_q_blocks + 1], kv_block_indices int32 [nnz], ascending and unique inside a row.
  *   - Execution order: row_order int32 [heads][n_q_blocks]; row_order[h][p] is the query
  *     block executed at position p of head h (the index-list form of P_h in Algorithm 2).
+ *
+ * Shape of the interface (choices of this library, fixed here so that callers need not guess)
+ *   - batch is flattened into `heads`, so strides have two entries {head, token};
+ *   - bf16 is the only element type, so there is no dtype field;
+ *   - a plan call's outputs are grouped in one struct, waveal_plan_out: one required, the rest optional;
+ *   - workspace sizes depend on the descriptor alone, never on the number of selected blocks;
+ *   - dev_status has four int32 words {code, site, head or block, value};
+ *   - a workspace is state of the call that uses it: two calls that may overlap on the GPU
+ *     (different streams or host threads) need a workspace each.
  */
 #ifndef WAVEAL_H_
 #define WAVEAL_H_
@@ -154,9 +163,15 @@ size_t waveal_noalloc_max_rows(void);
  * paper's backends apply it) in a single launch.  Without the flag the kernel fixes each row's
  * reference after the first two blocks of a task - softmax does not depend on the reference as
  * long as nothing overflows - watches the size of every block's sum, lists the tasks where a
- * sum reached 2^80 and computes those again, with the max of every block, in a second launch
+ * sum reached 2^24 and computes those again, with the max of every block, in a second launch
  * on the same stream.  Results agree to rounding; the flag exists for comparison runs. */
 #define WAVEAL_ATTN_ONLINE_MAX_ONLY 1
+/* Self-test of the kernel's failure handling, never set in production: the loader leaves out
+ * the first K tile of the first task and every bounded wait gives up after about 2 ms instead
+ * of 2 s.  The call must come back with dev_status = {WAVEAL_ERR_TIMEOUT, site 12, ...}, all
+ * thread blocks leaving through the common exit (no trap, no fault, the context stays usable);
+ * O is then undefined.  The next call on the same workspace works as usual. */
+#define WAVEAL_ATTN_SELFTEST_LOST_TILE 256
 
 typedef struct waveal_attn_desc {
   int32_t heads;            /* batch*heads; K/V heads == Q heads                              */
@@ -166,13 +181,16 @@ typedef struct waveal_attn_desc {
   int64_t q_stride[2], k_stride[2], v_stride[2], o_stride[2]; /* elements: {head, token}; head_dim contiguous */
   int32_t order_heads_interleaved; /* 0 = heads run one after another (Section 5, sequential
                                       heads); 1 = position-major across heads (parallel heads) */
-  int32_t flags;            /* 0, or WAVEAL_ATTN_ONLINE_MAX_ONLY                               */
+  int32_t flags;            /* 0, or WAVEAL_ATTN_* bits                                        */
 } waveal_attn_desc;
 
 /* Bytes of device workspace waveal_bsattn_fwd needs: 32 bytes of counters (int32 words: ticket
- * counter, abort flag, number of tasks computed twice, ticket counter of the second launch),
- * 8 bytes per (head, query block) for the list of tasks to compute again and 32 bytes per
- * (head, query block) for the table that maps a ticket to its task.  Host-only. */
+ * counter, abort flag, number of tasks computed twice, ticket counter of the second launch,
+ * length of the first and of the second launch in SM cycles = the largest lifetime of a thread
+ * block, two spare), 8 bytes per (head, query block) for the list of tasks to compute again and
+ * 32 bytes per (head, query block) for the table that maps a ticket to its task.  The counters
+ * are live state of the call (tickets are drawn from them): calls that may overlap on the GPU
+ * must not share a workspace.  Host-only. */
 waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* desc /*host*/, size_t* bytes /*host*/);
 
 /* Block-sparse attention forward, bf16 in / fp32 accumulate / bf16 out (Sections 2.1-2.3):
@@ -186,10 +204,18 @@ waveal_status waveal_bsattn_workspace_bytes(const waveal_attn_desc* desc /*host*
  * lse: dev float [heads][seq_q] or NULL (natural-log sum-exp per query token; -inf for a
  * query block with an empty list, whose O is 0).
  * scale <= 0 means 1/sqrt(head_dim).
- * ws: dev workspace (waveal_bsattn_workspace_bytes), 16-byte aligned; after the call its int32
- * word 2 holds the number of tasks the second launch computed again (normally 0).
- * dev_status: dev int32 [4] or NULL: {code, site, block, aux}; written only on a device-side
- * failure (the caller zeroes it).
+ * ws: dev workspace (waveal_bsattn_workspace_bytes), 16-byte aligned, not shared with a call
+ * that may run at the same time; after the call its int32 word 2 holds the number of tasks the
+ * second launch computed again (normally 0) and word 4 the launch's length in SM cycles.
+ * dev_status: dev int32 [4] or NULL, zeroed by the caller; written only on a device-side
+ * failure: {WAVEAL_ERR_TIMEOUT, site of the wait, thread block, thread} when a bounded wait ran
+ * out, {WAVEAL_ERR_BAD_MASK, site, head, value} for an entry of row_order outside [0, M_B)
+ * (site 31), a row-pointer pair that is negative, decreasing or beyond kv_row_ptr's last
+ * entry (32), or an index outside [0, N_B) (33: last of a list, 30: any other, met while
+ * loading).  A task with a bad row pointer or last index gets an empty list (its rows of O
+ * become 0); a bad index inside a list is replaced by block 0; the kernel never reads out of
+ * range.  row_order is not checked for being a permutation: a query block named twice is
+ * computed twice, one never named keeps its old contents.
  * The first call in a process also looks up a driver entry point (no allocation). */
 waveal_status waveal_bsattn_fwd(const waveal_attn_desc* desc /*host*/, const void* Q, const void* K, const void* V,
                                 void* O, float* lse, const int32_t* kv_row_ptr /*dev*/,

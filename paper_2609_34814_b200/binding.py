@@ -246,6 +246,7 @@ def scatter_rows(src, dst, row_order, block: int, stream=None):
 
 
 ATTN_ONLINE_MAX_ONLY = 1
+ATTN_SELFTEST_LOST_TILE = 256
 
 
 def attn_desc(q, k, v, o, seq_q: int, seq_kv: int, block: int, interleaved: bool = False, flags: int = 0) -> AttnDesc:

@@ -29,6 +29,7 @@ def measure(cfg, reps: int):
     import torch
     from . import binding as wb
     from . import inputs as I
+    from . import timing as wt
 
     dev = torch.device("cuda")
     H, S, Sp, D, B, nb = cfg.heads, cfg.seq, cfg.seq_pad, cfg.head_dim, cfg.block, cfg.n_blocks
@@ -62,12 +63,22 @@ def measure(cfg, reps: int):
 
     plan = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream)
     t_plan = timed(lambda: wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream))
-    t_nat = timed(lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=None, workspace=aws, dev_status=st, stream=stream))
-    t_reo = timed(lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=plan.row_order, workspace=aws, dev_status=st, stream=stream))
+    # the two orders alternate launch by launch (a drifting SM clock then hits both alike); the
+    # gain is taken from the median per-pair ratio, and the kernel's own cycle counts give the
+    # clock-independent view
+    aws_words = aws.view(torch.int32)
+    ab = wt.ab_interleaved(
+        lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=plan.row_order, workspace=aws, dev_status=st, stream=stream),
+        lambda: wb.bsattn_fwd(adesc, q, k, v, o, ptr, idx, row_order=None, workspace=aws, dev_status=st, stream=stream),
+        reps, stream, cycles_of=lambda: aws_words[4:5])
     if st.tolist()[0] != 0:
         raise RuntimeError(f"attention kernel reported {st.tolist()}")
+    t_reo = ab["a_ms"]
+    t_nat = t_reo * ab["b_over_a"]
     return {"frames": cfg.frames, "seq": S, "density": pairs / (H * nb * nb), "pairs": pairs,
             "kv_bytes_per_head": 2 * Sp * D * 2, "natural_ms": t_nat, "planned_ms": t_reo, "plan_ms": t_plan,
+            "natural_over_planned": ab["b_over_a"], "ratio_min": ab["b_over_a_min"], "ratio_max": ab["b_over_a_max"],
+            "natural_over_planned_cycles": ab.get("b_over_a_cycles"),
             "gain_ms": t_nat - t_reo - t_plan, "pays": bool(t_nat - t_reo > t_plan)}
 
 
@@ -78,7 +89,8 @@ def main(argv=None):
                          "while the attention time grows with the heads - calibrate at the deployment's head count")
     ap.add_argument("--frames", default="11,21,41,61,101")
     ap.add_argument("--densities", default="0.02,0.04,0.10")
-    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--reps", type=int, default=8, help="interleaved launch pairs per grid point")
+    ap.add_argument("--recipe", default="long720p", help="config whose mask recipe the grid scales (long720p, wan720p)")
     ap.add_argument("--json", default="")
     args = ap.parse_args(argv)
     import torch
@@ -89,7 +101,7 @@ def main(argv=None):
         raise RuntimeError("the guard is calibrated on the device it will run on: a CUDA device is required")
     wb.load()
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    base = I.CONFIGS["long720p"]
+    base = I.CONFIGS[args.recipe]
     rows = []
     for fr in (int(x) for x in args.frames.split(",")):
         for rho in (float(x) for x in args.densities.split(",")):
@@ -97,9 +109,12 @@ def main(argv=None):
             r = measure(cfg, args.reps)
             r["kv_over_l2"] = r["kv_bytes_per_head"] / l2
             rows.append(r)
-            print("frames %4d  seq %7d  density %.3f  K+V/L2 %.2f  natural %8.3f  planned %8.3f  plan %6.3f  gain %+7.3f ms  %s"
-                  % (fr, r["seq"], r["density"], r["kv_over_l2"], r["natural_ms"], r["planned_ms"], r["plan_ms"],
-                     r["gain_ms"], "pays" if r["pays"] else "skip"), flush=True)
+            print("frames %4d  seq %7d  density %.3f  K+V/L2 %.2f  natural %8.3f  planned %8.3f  ratio %.3f [%.3f, %.3f] cycles %s  "
+                  "plan %6.3f  gain %+7.3f ms  %s"
+                  % (fr, r["seq"], r["density"], r["kv_over_l2"], r["natural_ms"], r["planned_ms"], r["natural_over_planned"],
+                     r["ratio_min"], r["ratio_max"],
+                     "%.3f" % r["natural_over_planned_cycles"] if r["natural_over_planned_cycles"] else "-",
+                     r["plan_ms"], r["gain_ms"], "pays" if r["pays"] else "skip"), flush=True)
     # thresholds: the largest K+V/L2 ratio at which planning never paid, and the largest density
     # at which it never paid once K+V no longer fits
     never = [r["kv_over_l2"] for r in rows if not any(x["pays"] for x in rows if x["frames"] == r["frames"])]

@@ -27,7 +27,7 @@
 //               inverse permutation)
 // Two launches per call: in the first the row max is taken in blocks 0 and 1 of a task only and
 // the reference stays fixed afterwards (softmax does not depend on it short of overflow); a task
-// in which a block's sum of exponentials reaches 2^80 is listed in the workspace and computed
+// in which a block's sum of exponentials reaches 2^24 is listed in the workspace and computed
 // again by the second launch, which takes the max of every block.
 // Every wait on an mbarrier is bounded; when one runs out the CTA records
 // {WAVEAL_ERR_TIMEOUT, site} and all roles leave through the common teardown.
@@ -41,6 +41,7 @@ namespace {
 constexpr int kThreads = 352;
 constexpr int kProducerWarp = 0, kPvWarp = 1, kSoftmaxWarp0 = 2, kQkWarp = 10;
 constexpr long long kTimeoutCycles = 4000000000ll;   // ~2 s at boost clock
+constexpr long long kSelfTestCycles = 4000000ll;     // ~2 ms: wait limit under WAVEAL_ATTN_SELFTEST_LOST_TILE
 #ifndef WAVEAL_POLY_EVERY
 #define WAVEAL_POLY_EVERY 2
 #endif
@@ -148,18 +149,32 @@ __device__ __forceinline__ void fadd2(float& d0, float& d1, float a0, float a1, 
       : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
 }
 
-// 2^x for two values on the FMA and integer pipes (for a share of the elements, to take load
+// 2^(x) for two values on the FMA and integer pipes (for a share of the elements, to take load
 // off the transcendental unit: at 16 results per clock and SM it is as busy as the tensor
-// cores): x is rounded to the nearest integer n with the 1.5*2^23 trick, a degree-3 polynomial
-// gives 2^(x-n) on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16 cut of P), and n is
-// added to the exponent field.  Multiply-adds work on register pairs.
-__device__ __forceinline__ void ex2_fma2(float& e0, float& e1, float x0, float x1) {
-  x0 = fmaxf(x0, -125.0f);
-  x1 = fmaxf(x1, -125.0f);
+// cores).  The caller passes s and the pair (a, b) of x = a*s + b.  The argument is first
+// confined to the window [kPolyLo, kPolyLo + 128] by a saturating multiply-add
+// (y = sat(x/128 - kPolyLo/128) in [0, 1]; x is taken back from y with an absolute error
+// below 2^-17), so that the exponent arithmetic below can neither wrap into the sign bit
+// (x >= 128.5 would) nor underflow: an x above the window comes out as 2^(kPolyLo+128) = 2^28,
+// far above the limit at which the fixed-reference pass hands a task to the second launch; an x
+// below it (a key that does not exist, -inf) as 2^-100.  x is then rounded to the nearest integer
+// n with the 1.5*2^23 trick, a degree-3 polynomial gives 2^(x-n) on [-0.5, 0.5] (relative error
+// 7.5e-5, far below the bf16 cut of P), and n is added to the exponent field.
+constexpr float kPolyLo = -100.0f;
+constexpr float kRedoLimit = 16777216.0f;     // 2^24: block sums at or above it (or NaN) list the task
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {
+  float d;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ void ex2_fma2(float& e0, float& e1, float s0, float s1, float a128, float b128) {
+  // a128 = a/128, b128 = (b - kPolyLo)/128
+  const float y0 = fma_sat(s0, a128, b128), y1 = fma_sat(s1, a128, b128);
+  constexpr float kMagic = 12582912.0f;                 // 1.5 * 2^23
   float xi0, xi1, n0, n1, f0, f1, q0, q1;
-  fadd2(xi0, xi1, x0, x1, 12582912.0f, 12582912.0f);
-  fadd2(n0, n1, xi0, xi1, -12582912.0f, -12582912.0f);
-  ffma2(f0, f1, n0, n1, -1.0f, -1.0f, x0, x1);
+  ffma2(xi0, xi1, y0, y1, 128.0f, 128.0f, kMagic + kPolyLo, kMagic + kPolyLo);   // bits: 0x4B400000 + n
+  fadd2(n0, n1, xi0, xi1, -(kMagic + kPolyLo), -(kMagic + kPolyLo));             // n - kPolyLo = round(128 y)
+  ffma2(f0, f1, y0, y1, 128.0f, 128.0f, -n0, -n1);                               // x - n
   ffma2(q0, q1, f0, f1, 0.05517137423157692f, 0.05517137423157692f, 0.2426110953092575f, 0.2426110953092575f);
   ffma2(q0, q1, q0, q1, f0, f1, 0.6932610273361206f, 0.6932610273361206f);
   ffma2(q0, q1, q0, q1, f0, f1, 0.9999280571937561f, 0.9999280571937561f);
@@ -213,16 +228,9 @@ __device__ __forceinline__ void ex2_fma2(float& e0, float& e1, float x0, float x
       : "memory")
 
 __device__ __forceinline__ float ex2(float x) {
-#ifdef WAVEAL_DBG_NOEXP
-  return x * 0.001f + 0.5f;
-#else
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-#endif
-}
-__device__ __forceinline__ void named_bar_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 // shared-memory matrix descriptor, 128-byte swizzle, Blackwell version field
@@ -261,6 +269,8 @@ struct AttnParams {
   long long o_stride_h, o_stride_t;
   int heads, m_b, n_b, seq_q, seq_kv, interleaved;
   long long total_tasks;
+  long long wait_limit;   // cycles a bounded wait may take (kTimeoutCycles; far shorter under the self-test flag)
+  int drop_tile;          // self-test: the producer never loads the first K tile of ticket 0
   float sl2;          // scale * log2(e)
 };
 
@@ -273,11 +283,7 @@ struct Geo {
   static constexpr int TILE_BYTES = SLABS * BK * 128;
   static constexpr int KV_SLAB_BYTES = BK * 128;
   static constexpr int NSTAGE_RAW = (200 * 1024 - Q_BYTES) / TILE_BYTES;
-#ifdef WAVEAL_DBG_NSTAGE
-  static constexpr int NSTAGE = WAVEAL_DBG_NSTAGE;
-#else
   static constexpr int NSTAGE = NSTAGE_RAW > 8 ? 8 : NSTAGE_RAW;
-#endif
   static constexpr int NKS = (NSTAGE + 1) / 2;       // K tile ring
   static constexpr int NVS = NSTAGE / 2;             // V tile ring
   static constexpr int NSBUF = 3;                    // S/P buffers in tensor memory
@@ -288,7 +294,7 @@ struct Geo {
   static constexpr int OFF_K = OFF_Q + Q_BYTES;
   static constexpr int OFF_V = OFF_K + NKS * TILE_BYTES;
   static constexpr int OFF_BAR = OFF_V + NVS * TILE_BYTES;
-  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 4 * NSBUF + 2 + 1 + 8;
+  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 4 * NSBUF + 2 + 2 + 8 + 4;
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
   static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
   static constexpr int OFF_MISC = OFF_MX + 2 * 128 * 4 + 2 * 2 * 128 * 8;
@@ -297,27 +303,12 @@ struct Geo {
   static constexpr uint32_t S_STRIDE = 128, O_COL = 384, TMEM_COLS = 512;
 };
 
-#ifdef WAVEAL_TRACE
-// debug build only: four tracer threads of CTA 0 append (tag, block, clock) records to their own
-// region after the 256-byte workspace header (plain stores, no atomics)
-#define TRACE_DECL int trace_n_ = 0
-#define TRACE(role, tag, j)                                                                    \
-  do {                                                                                         \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && trace_n_ < 4000) {                       \
-      int* r_ = p.ws + 64 + (role) * 8000 + 2 * trace_n_;                                      \
-      r_[0] = (tag) | ((j) << 8); r_[1] = (int)clock64(); ++trace_n_;                          \
-    }                                                                                          \
-  } while (0)
-#else
-#define TRACE_DECL
-#define TRACE(role, tag, j) do {} while (0)
-#endif
-
 struct Ctx {
   uint32_t bar_base;
   volatile int* abort_smem;
   int* ws;
   int* dev_status;
+  long long limit;      // cycles a wait may take before the CTA gives up
 };
 
 __device__ __noinline__ void signal_abort(const Ctx& c, int site) {
@@ -339,7 +330,7 @@ __device__ __forceinline__ bool mbar_wait(const Ctx& c, uint32_t bar, uint32_t p
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*c.abort_smem) return false;
-    if (clock64() - t0 > kTimeoutCycles) { signal_abort(c, site); return false; }
+    if (clock64() - t0 > c.limit) { signal_abort(c, site); return false; }
   }
 }
 
@@ -369,15 +360,17 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   constexpr int B_TASK_FULL = 0, B_TASK_EMPTY = 2, B_Q_FULL = 4, B_Q_EMPTY = 5, B_K_FULL = 6,
                 B_K_EMPTY = B_K_FULL + G::NKS, B_V_FULL = B_K_EMPTY + G::NKS, B_V_EMPTY = B_V_FULL + G::NVS,
                 B_S_FULL = B_V_EMPTY + G::NVS, B_P_FULL = B_S_FULL + G::NSBUF, B_S_FREE = B_P_FULL + 2 * G::NSBUF,
-                B_O_FULL = B_S_FREE + G::NSBUF, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1, B_MX = B_FINAL + 1;
-  static_assert(B_MX + 8 <= G::N_BAR, "barrier count");
+                B_O_FULL = B_S_FREE + G::NSBUF, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1, B_MX = B_FINAL + 2,
+                B_EX = B_MX + 8;
+  static_assert(B_EX + 4 <= G::N_BAR, "barrier count");
   Task* tasks = reinterpret_cast<Task*>(smem + G::OFF_TASK);
   volatile float* mpub = reinterpret_cast<volatile float*>(smem + G::OFF_MX);   // [block parity][128] reference max after a block
   float2* ex = reinterpret_cast<float2*>(smem + G::OFF_MX + 2 * 128 * 4);       // [task parity][team][128] (reference, sum)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + G::OFF_MISC);
   volatile int* abort_smem = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 4);
   volatile int* redo_flag = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 8);   // [task parity]
-  Ctx ctx{bar0, abort_smem, p.ws, p.dev_status};
+  Ctx ctx{bar0, abort_smem, p.ws, p.dev_status, p.wait_limit};
+  const long long t_start = clock64();
 
   if (tid == 0) {
     // a task is read by the two MMA issuers and the eight softmax warps
@@ -395,7 +388,9 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     mbar_init(BAR(B_O_FULL), 1);
     mbar_init(BAR(B_O_FREE), 8);
     mbar_init(BAR(B_FINAL), 1);
+    mbar_init(BAR(B_FINAL + 1), 1);
     for (int i = 0; i < 8; ++i) mbar_init(BAR(B_MX + i), 1);
+    for (int i = 0; i < 4; ++i) mbar_init(BAR(B_EX + i), 2);    // the two warps of a lane quadrant, once per task
     *abort_smem = 0;
     redo_flag[0] = 0;
     redo_flag[1] = 0;
@@ -479,25 +474,28 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           my_idx = q < tk.n ? p.kv_idx[tk.lo + q] : 0;
         }
         int blk = __shfl_sync(0xffffffffu, my_idx, j - chunk_base);
-        if (blk < 0 || blk >= p.n_b) blk = 0;            // malformed list: stay in range
+        if (blk < 0 || blk >= p.n_b) {                   // malformed list: report it and stay in range
+          if (lane == 0 && p.dev_status && atomicCAS(p.dev_status, 0, WAVEAL_ERR_BAD_MASK) == 0) {
+            p.dev_status[1] = 30; p.dev_status[2] = tk.h; p.dev_status[3] = blk;
+          }
+          blk = 0;
+        }
         const uint32_t it = is_k ? k_it : v_it;
         const uint32_t nst = is_k ? (uint32_t)G::NKS : (uint32_t)G::NVS;
         const uint32_t st = it % nst, sph = (it / nst) & 1;
         const int b_full = (is_k ? B_K_FULL : B_V_FULL) + (int)st, b_empty = (is_k ? B_K_EMPTY : B_V_EMPTY) + (int)st;
         if (!warp_wait(ctx, BAR(b_empty), sph ^ 1, 3)) return false;
-        if (lane == 0) {
-#ifdef WAVEAL_DBG_NOLOAD
-          if (it >= nst) { mbar_arrive(BAR(b_full)); } else
-#endif
-          {
+        // (self-test of the abort path: one tile is never requested, so its consumer's wait runs out)
+        const bool dropped = p.drop_tile && is_k && t == 0 && j == 0;
+        if (lane == 0 && !dropped) {
           mbar_expect_tx(BAR(b_full), G::TILE_BYTES);
           const CUtensorMap* tm = is_k ? &tmK : &tmV;
           const uint32_t dst = sbase + (is_k ? G::OFF_K : G::OFF_V) + st * G::TILE_BYTES;
 #pragma unroll
           for (int s = 0; s < G::SLABS; ++s)
             tma_load_3d(dst + s * G::KV_SLAB_BYTES, tm, s * 64, blk * G::BK, tk.h, BAR(b_full));
-          }
         }
+        if (dropped) { ++k_it; return true; }
         if (is_k) { k_armed |= 1u << st; k_parity = (k_parity & ~(1u << st)) | (sph << st); ++k_it; }
         else { v_armed |= 1u << st; v_parity = (v_parity & ~(1u << st)) | (sph << st); ++v_it; }
         return true;
@@ -513,16 +511,16 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       for (int st = 0; st < G::NKS; ++st)
         if (k_armed & (1u << st)) {
           long long t0 = clock64();
-          while (!mbar_try_wait(BAR(B_K_FULL + st), (k_parity >> st) & 1) && clock64() - t0 < kTimeoutCycles / 4) {}
+          while (!mbar_try_wait(BAR(B_K_FULL + st), (k_parity >> st) & 1) && clock64() - t0 < p.wait_limit / 4) {}
         }
       for (int st = 0; st < G::NVS; ++st)
         if (v_armed & (1u << st)) {
           long long t0 = clock64();
-          while (!mbar_try_wait(BAR(B_V_FULL + st), (v_parity >> st) & 1) && clock64() - t0 < kTimeoutCycles / 4) {}
+          while (!mbar_try_wait(BAR(B_V_FULL + st), (v_parity >> st) & 1) && clock64() - t0 < p.wait_limit / 4) {}
         }
       if (q_armed) {
         long long t0 = clock64();
-        while (!mbar_try_wait(BAR(B_Q_FULL), q_armed_parity) && clock64() - t0 < kTimeoutCycles / 4) {}
+        while (!mbar_try_wait(BAR(B_Q_FULL), q_armed_parity) && clock64() - t0 < p.wait_limit / 4) {}
       }
     }
   } else if (warp == kQkWarp) {
@@ -535,7 +533,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     // (shuffle-broadcast values, compare-and-reset ring positions).
     constexpr uint32_t IDESC_QK = make_idesc(128, G::BK, false);
     uint32_t task_slot = 0, task_ph = 0, q_ph = 0, k_st = 0, k_ph = 0, sb = 0, free_bits = 0, first_uses = G::NSBUF;
-    TRACE_DECL;
     const uint64_t qdesc0 = make_desc(sbase + G::OFF_Q, 16, 1024);
     const uint64_t kdesc0 = make_desc(sbase + G::OFF_K, 16, 1024);
     bool ok = true;
@@ -564,7 +561,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           if (!ok) break;
         }
         free_bits ^= 1u << sb;
-        TRACE(3, 4, j);
         tc_fence_after();
         {
           // descriptors differ from the per-kernel bases only in the 14-bit address field
@@ -572,25 +568,29 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           const uint32_t d_s = tmem_base + sb * G::S_STRIDE;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
-#ifndef WAVEAL_DBG_SKIP_QK
             umma_bf16(d_s, qdesc0 + (uint64_t)(((k / 4) * 128 * 128 + (k % 4) * 32) >> 4),
                       kd + (uint64_t)(((k / 4) * G::KV_SLAB_BYTES + (k % 4) * 32) >> 4), IDESC_QK, k > 0);
-#endif
           }
           tc_commit(BAR(B_K_EMPTY + k_st));
           tc_commit(BAR(B_S_FULL + sb));
           if (j == n - 1) tc_commit(BAR(B_Q_EMPTY));
         }
-        TRACE(3, 5, j);
         if (++k_st == (uint32_t)G::NKS) { k_st = 0; k_ph ^= 1; }
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
+    }
+    // none of this thread's MMAs is still running when tensor memory is released (in a regular
+    // run the last P V already depends on all of them; after an abort nothing else orders them)
+    tc_commit(BAR(B_FINAL + 1));
+    __syncwarp();
+    {
+      long long t0 = clock64();
+      while (!mbar_try_wait(BAR(B_FINAL + 1), 0) && clock64() - t0 < p.wait_limit / 4) {}
     }
   } else if (warp == kPvWarp) {
     // ============================================================== MMA issuer 2: O += P V
     constexpr uint32_t IDESC_PV = make_idesc(128, D, true);
     uint32_t task_slot = 0, task_ph = 0, o_ph = 1, v_st = 0, v_ph = 0, sb = 0, p_phase = 0;
-    TRACE_DECL;
     const uint64_t vdesc0 = make_desc(sbase + G::OFF_V, G::KV_SLAB_BYTES, 1024);
     bool ok = true;
     while (ok) {
@@ -621,10 +621,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           if (!ok) break;
           p_phase ^= 1u << pb;
           if (h == 0) {
-            TRACE(0, 1, j);
             ok = warp_wait(ctx, BAR(B_V_FULL + v_st), v_ph, 15);
             if (!ok) break;
-            TRACE(0, 2, j);
           }
           tc_fence_after();
           // V tile as the N x K operand with N (head_dim) contiguous: 8 keys per 1024-byte
@@ -632,9 +630,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #pragma unroll
           for (int kk = 0; kk < G::BK / 32; ++kk) {
             const int k = h * (G::BK / 32) + kk;
-#ifndef WAVEAL_DBG_SKIP_PV
             umma_bf16_ts(d_o, pbase + k * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
-#endif
           }
         }
         if (!ok) break;
@@ -643,7 +639,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           tc_commit(BAR(B_S_FREE + sb));
           if (j == n - 1) tc_commit(BAR(B_O_FULL));
         }
-        TRACE(0, 3, j);
         if (++v_st == (uint32_t)G::NVS) { v_st = 0; v_ph ^= 1; }
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
@@ -654,7 +649,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     __syncwarp();
     {
       long long t0 = clock64();
-      while (!mbar_try_wait(BAR(B_FINAL), 0) && clock64() - t0 < kTimeoutCycles / 4) {}
+      while (!mbar_try_wait(BAR(B_FINAL), 0) && clock64() - t0 < p.wait_limit / 4) {}
     }
   } else {
     // ============================================================== softmax / epilogue
@@ -674,7 +669,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t o_row = tmem_base + lane_addr + G::O_COL;
     uint32_t task_it = 0, s_phase = 0, o_it = 0, mx_phase = 0, sb = 0;   // s_phase bit b: parity of the uses of S[b] so far
-    TRACE_DECL;
     bool ok = true;
     while (ok) {
       const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
@@ -705,17 +699,15 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if ((int)par == team) {
           ok = warp_wait(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
           if (!ok) break;
-          if (quad == 2) TRACE(1 + team, 10 + team, j);
           tc_fence_after();
           const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE;
           const bool ragged = j == tk.n - 1 && tk.tail_valid < G::BK;
-#ifndef WAVEAL_DBG_NOSM   // (timing experiments only: with the macro the softmax warps just pass the barriers on)
           // ---- pass 1: row max (the values are loaded again for the exponentials: a second
           // tensor-memory load is cheaper than 128 live registers)
           // In the first pass over the tasks (FAST) only blocks 0 and 1 of a task take a max and
           // may move the reference; from block 2 on both teams keep the reference of block 1.
           // Any reference gives the same softmax as long as nothing overflows, so the later
-          // blocks only watch the largest exponent they produce: if it ever exceeds 100 the
+          // blocks only watch the sum of the exponentials they produce: if it ever reaches 2^24 the
           // task is put on a list and computed again by the second launch, which takes the
           // max of every block (the rule of the paper's online softmax).
           const bool fixed_ref = FAST && j >= 2;
@@ -745,7 +737,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             mloc = fmaxf(mloc, fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
                                      fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7]))));
           }
-          if (quad == 2) TRACE(1 + team, 12 + team, j);
           // ---- the row's reference after block j-1, from the other team
           float m_prev = m_ref;
           if (j > 0 && (!fixed_ref || j == 2)) {
@@ -793,6 +784,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           // around zero, like a rounding; the row sum adds the uncut p' and the epilogue takes
           // the factor out again.  Multiply-adds and sums work on register pairs (f32x2).
           const float neg_m = ((m_new == -INFINITY) ? 0.f : -m_new) + 0.0028150156f;
+          const float a128 = p.sl2 * 0.0078125f, b128 = (neg_m - kPolyLo) * 0.0078125f;   // polynomial share
           float ls4[4] = {0.f, 0.f, 0.f, 0.f};
           // ---- pass 2: exponentials; P_j (bf16 pairs) goes over the first half of the row's own
           // S columns, each chunk after its S values have been read
@@ -811,12 +803,12 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             uint32_t pk[G::CH / 2];
 #pragma unroll
             for (int c = 0; c < G::CH; c += 2) {
-              float x0, x1;
-              ffma2(x0, x1, __uint_as_float(sv[c]), __uint_as_float(sv[c + 1]), p.sl2, p.sl2, neg_m, neg_m);
               float e0, e1;
               if (kPolyEvery > 0 && ((c >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == (kPolyEvery > 0 ? kPolyEvery : 1) - 1) {
-                ex2_fma2(e0, e1, x0, x1);
+                ex2_fma2(e0, e1, __uint_as_float(sv[c]), __uint_as_float(sv[c + 1]), a128, b128);
               } else {
+                float x0, x1;
+                ffma2(x0, x1, __uint_as_float(sv[c]), __uint_as_float(sv[c + 1]), p.sl2, p.sl2, neg_m, neg_m);
                 e0 = ex2(x0); e1 = ex2(x1);
               }
               fadd2(ls4[c & 2], ls4[(c & 2) + 1], ls4[c & 2], ls4[(c & 2) + 1], e0, e1);
@@ -834,16 +826,11 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           }
           const float l_blk = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
           l_run += l_blk;
-          // all terms are positive, so a block sum below 2^80 bounds every exponent of the block;
-          // above it (or not a number) the fixed reference is too far off: redo the task
-          if (fixed_ref && __any_sync(0xffffffffu, !(l_blk < 1.2089258e24f))) redo_flag[rslot] = 1;
-          if (quad == 2) TRACE(1 + team, 14 + team, j);
-#else
-          if (j > 0) { ok = warp_wait(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24); if (!ok) break; }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(BAR(B_MX + quad * 2 + par));
-          l_run = 1.f; m_ref = 0.f;
-#endif
+          // all terms are positive (the transcendental unit returns +inf on overflow, the
+          // polynomial share saturates at 2^28), so a block sum below 2^24 bounds every exponent
+          // of the block; at or above it (or not a number) the fixed reference is too far off:
+          // redo the task
+          if (fixed_ref && __any_sync(0xffffffffu, !(l_blk < kRedoLimit))) redo_flag[rslot] = 1;
           tc_wait_st();
           tc_fence_before();
           __syncwarp();
@@ -851,7 +838,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             if (G::NCH != 2) mbar_arrive(BAR(B_P_FULL + sb * 2));
             mbar_arrive(BAR(B_P_FULL + sb * 2 + 1));
           }
-          if (quad == 2) TRACE(1 + team, 16 + team, j);
         }
         // both teams count every block
         s_phase ^= 1u << sb;
@@ -865,7 +851,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (!ok) break;
       ++o_it;
       tc_fence_after();
-      if (quad == 2) TRACE(1 + team, 18 + team, tk.n);
       if (FAST && sw == 0 && lane == 0 && redo_flag[rslot]) {
         // every warp's blocks of this task lie before O_FULL; the slot is used again two tasks
         // later, after this warp's O_FREE arrival below
@@ -875,7 +860,12 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         redo_flag[rslot] = 0;
       }
       exb[team * 128 + r] = make_float2(m_ref, l_run);
-      named_bar_sync(1 + quad, 64);
+      // the partner warp of this lane quadrant (other team) has written its half: a bounded wait
+      // like every other, so that a warp whose partner gave up does not stay behind
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_EX + quad));
+      ok = warp_wait(ctx, BAR(B_EX + quad), (o_it & 1) ^ 1, 25);
+      if (!ok) break;
       const float2 oth = exb[(team ^ 1) * 128 + r];
       const float m_all = fmaxf(m_ref, oth.x);
       const float a_self = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_all);
@@ -890,7 +880,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_O_FREE));
-      if (quad == 2) TRACE(1 + team, 30 + team, tk.n);
       if (row_live) {
 #pragma unroll
         for (int c = 0; c < G::CO; c += 8) {
@@ -915,24 +904,47 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     tc_fence_after();
     tmem_dealloc(tmem_base, G::TMEM_COLS);
   }
+  // SM cycles this CTA was alive: the largest over the grid is the launch's length in cycles,
+  // a figure that does not depend on the clock the GPU happened to run at
+  if (tid == 0) {
+    const long long dt = clock64() - t_start;
+    atomicMax(&p.ws[p.redo_pass ? 5 : 4], (int)(dt > 0x7fffffffll ? 0x7fffffffll : dt));
+  }
 }
 
 // Task of every ticket (head-major or position-major over the planned order), so that the
 // persistent CTAs need one load behind a ticket instead of a chain through row_order, the row
 // pointers and the index list.
+// The inputs are checked on the way (one thread per task, so it costs nothing): an entry of
+// row_order outside [0, M_B), a row-pointer pair that is negative, decreasing or beyond the end
+// of the index list, or a last index outside [0, N_B) is reported as
+// {WAVEAL_ERR_BAD_MASK, site, head, offending value} and the task is given an empty list
+// (its output rows become 0) instead of reading out of range.
 __global__ void k_task_table(AttnParams p, int block_k, Task* table) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= p.total_tasks) return;
   int h, pos;
   if (p.interleaved) { pos = (int)(t / p.heads); h = (int)(t % p.heads); }
   else { h = (int)(t / p.m_b); pos = (int)(t % p.m_b); }
+  auto report = [&](int site, int value) {
+    if (p.dev_status && atomicCAS(p.dev_status, 0, WAVEAL_ERR_BAD_MASK) == 0) {
+      p.dev_status[1] = site; p.dev_status[2] = h; p.dev_status[3] = value;
+    }
+  };
   int row = p.row_order ? p.row_order[(size_t)h * p.m_b + pos] : pos;
-  if (row < 0 || row >= p.m_b) row = pos;          // never index out of range
+  bool bad = false;
+  if (row < 0 || row >= p.m_b) { report(31, row); row = pos; bad = true; }
+  const long long nnz = p.row_ptr[p.total_tasks];
   const int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
+  if (lo < 0 || hi < lo || (long long)hi > nnz) { report(32, lo < 0 ? lo : hi); bad = true; }
   Task tk{};
-  tk.h = h; tk.row = row; tk.lo = lo; tk.n = max(hi - lo, 0);
+  tk.h = h; tk.row = row; tk.lo = bad ? 0 : lo; tk.n = bad ? 0 : hi - lo;
   tk.tail_valid = block_k;
-  if (tk.n > 0 && (p.seq_kv % block_k) != 0 && p.kv_idx[hi - 1] == p.n_b - 1) tk.tail_valid = p.seq_kv % block_k;
+  if (tk.n > 0) {
+    const int last = p.kv_idx[hi - 1];
+    if (last < 0 || last >= p.n_b) { report(33, last); tk.n = 0; }
+    else if ((p.seq_kv % block_k) != 0 && last == p.n_b - 1) tk.tail_valid = p.seq_kv % block_k;
+  }
   table[t] = tk;
 }
 
@@ -1009,6 +1021,9 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   p.redo_pass = 0;
   k_task_table<<<(unsigned)((p.total_tasks + 255) / 256), 256, 0, st>>>(p, BLOCK, table);
   WAVEAL_CUDA_OK(cudaGetLastError());
+  p.wait_limit = kTimeoutCycles;
+  p.drop_tile = 0;
+  if (d->flags & WAVEAL_ATTN_SELFTEST_LOST_TILE) { p.wait_limit = kSelfTestCycles; p.drop_tile = 1; }
   if (d->flags & WAVEAL_ATTN_ONLINE_MAX_ONLY) {
     p.redo_pass = 0;
     k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);

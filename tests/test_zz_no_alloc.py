@@ -54,3 +54,26 @@ def test_noalloc_matches_the_workspace_entry_point_twice_in_a_row():
         assert torch.equal(ptr, ref_ptr) and torch.equal(idx, ref_idx)
         host_ptr, host_idx = I.masks_to_csr(masks)
         assert np.array_equal(ptr.cpu().numpy(), host_ptr) and np.array_equal(idx.cpu().numpy(), host_idx)
+
+
+@pytest.mark.gpu
+def test_noalloc_at_exactly_the_largest_accepted_size():
+    """heads * n_q_blocks == waveal_noalloc_max_rows(): the scan then writes its last partial sum
+    from the last int of the built-in array."""
+    import torch
+    heads, rows, cols = 3, 87381, 8
+    assert heads * rows == wb.noalloc_max_rows()
+    rng = np.random.default_rng(11)
+    mask = rng.random((heads, rows, cols)) < 0.4
+    words = np.zeros((heads, rows, 1), dtype=np.uint64)
+    for j in range(cols):
+        words[:, :, 0] |= mask[:, :, j].astype(np.uint64) << np.uint64(j)
+    bitmap = torch.from_numpy(words.view(np.int64)).cuda()
+    counts = mask.reshape(-1, cols).sum(axis=1)
+    exp_ptr = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    exp_idx = np.nonzero(mask.reshape(-1, cols))[1].astype(np.int32)
+    ptr = torch.full((heads * rows + 1,), -1, dtype=torch.int32, device="cuda")
+    idx = torch.full((int(exp_ptr[-1]),), -1, dtype=torch.int32, device="cuda")
+    wb.bitmap_to_csr_noalloc(bitmap, cols, ptr, idx)
+    torch.cuda.synchronize()
+    assert np.array_equal(ptr.cpu().numpy(), exp_ptr) and np.array_equal(idx.cpu().numpy(), exp_idx)
