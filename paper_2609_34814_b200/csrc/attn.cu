@@ -423,7 +423,9 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       long long t = 0, n_tasks = p.total_tasks;
       if (lane == 0) {
         if (p.redo_pass) n_tasks = min((long long)p.ws[2], p.total_tasks);   // written by the first pass
-        t = (p.ws[1] != 0) ? n_tasks : (long long)(unsigned)atomicAdd(&p.ws[p.redo_pass ? 3 : 0], 1);
+        // (volatile: another SM raises the flag while this kernel runs; a cached copy would hide it)
+        t = (*reinterpret_cast<volatile int*>(&p.ws[1]) != 0) ? n_tasks
+                                                             : (long long)(unsigned)atomicAdd(&p.ws[p.redo_pass ? 3 : 0], 1);
       }
       t = __shfl_sync(0xffffffffu, t, 0);
       n_tasks = __shfl_sync(0xffffffffu, n_tasks, 0);
