@@ -59,7 +59,21 @@ def ncu_counters(workload: str):
 
 # --------------------------------------------------------------------------- oracle legs
 
-def oracle_sample(cfg, target_s=12.0, n_heads=4):
+ORACLE_MODES = {"reorder": 1, "natural": 2, "auto": 0, "stage1": 3, "stage2": 4}
+
+
+def l2_bytes_of_device() -> int:
+    """L2 size the guard compares with (the device's when one is visible, else the B200's 126 MB)."""
+    try:
+        import torch
+        if torch.cuda.is_available():
+            return int(torch.cuda.get_device_properties(0).L2_cache_size)
+    except Exception:
+        pass
+    return 126 * 1024 * 1024
+
+
+def oracle_sample(cfg, target_s=12.0, n_heads=4, plan_mode="auto"):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload: the plan
     (NumPy, every step of Algorithm 1/2) of `n_heads` heads and the attention (C twin, OpenMP
     over query tokens) of query blocks drawn from those heads until about `target_s` seconds
@@ -77,7 +91,8 @@ def oracle_sample(cfg, target_s=12.0, n_heads=4):
     for h in heads:
         mk = I.make_mask(cfg, h)
         t0 = time.perf_counter()
-        wo.plan_head(mk, 148, 5, cfg.plan_seed, h, mode=wo.MODE_FORCE_REORDER)   # T = the library default
+        wo.plan_head(mk, 148, 5, cfg.plan_seed, h, mode=ORACLE_MODES[plan_mode],          # T = the library default
+                     guard={"kv_bytes_per_head": 2 * cfg.seq_pad * cfg.head_dim * 2, "l2_bytes": l2_bytes_of_device()})
         t_plan += time.perf_counter() - t0
         bits = [I.make_head_tensor(cfg, w, h).view(torch.int16).numpy().view(np.uint16) for w in "qkv"]
         data.append((mk, bits, rng.permutation(cfg.n_blocks)))
@@ -108,7 +123,7 @@ def run_reference(args, cfg):
         return
     vals, infos, times = [], None, []
     for i in range(args.warmup + args.steps):
-        v, info, t = oracle_sample(cfg, target_s=5.0, n_heads=1)
+        v, info, t = oracle_sample(cfg, target_s=5.0, n_heads=1, plan_mode=args.plan_mode)
         if i >= args.warmup:
             vals.append(v); times.append(t); infos = info
     value = float(np.mean(vals))
@@ -356,7 +371,8 @@ def run_waveal(args, cfg):
     achieved = flops / (attn_ms * 1e-3) / 1e12
     ctr = ncu_counters(cfg.name) if args.mask == "videomask" and not split else {}
     traffic = None
-    key = "natural" if args.plan_mode == "natural" else "reordered"
+    step_skipped = int((plan.skip_flags & 1).sum().item())      # heads the timed steps ran in natural order
+    key = "natural" if step_skipped == H else "reordered" if step_skipped == 0 else "mixed"
     if f"dram_read_bytes_{key}" in ctr and f"dram_write_bytes_{key}" in ctr:
         traffic = ctr[f"dram_read_bytes_{key}"] + ctr[f"dram_write_bytes_{key}"]
     clocks = sampler.summary("timed steps")
@@ -367,7 +383,7 @@ def run_waveal(args, cfg):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "heads": cfg.heads, "heads_per_rank": H, "head_dim": D, "seq": S, "block": B,
                    "block_pairs_rank0": pairs,
-                   "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode,
+                   "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode, "heads_in_natural_order": step_skipped,
                    "mask": args.mask, "head_order": args.head_order, "svd_iters": int(pdesc.svd_iters),
                    "step": "plan + attention", "l2": "inputs (Q,K,V,O %.1f GB per rank) larger than L2, no flush" %
                    (4 * H * Sp * D * 2 / 1e9),
@@ -397,7 +413,7 @@ def run_waveal(args, cfg):
         "e2e": e2e, "gpu_launches": launches["n"], "clocks": clocks,
     }
     if world == 1 and not args.no_cpu:
-        v, info, _ = oracle_sample(cfg)
+        v, info, _ = oracle_sample(cfg, plan_mode=args.plan_mode)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
                                 "sample": info["sample"]}
     else:
@@ -414,8 +430,9 @@ def main():
     ap.add_argument("--impl", default="waveal", choices=["waveal", "reference"])
     ap.add_argument("--config", default="wan720p")
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling / parity cases)")
-    ap.add_argument("--plan-mode", default="reorder", choices=["reorder", "natural", "auto", "stage1", "stage2"],
-                    help="which stages the plan of the timed step runs (Section 6.5 ablation); the headline is 'reorder'")
+    ap.add_argument("--plan-mode", default="auto", choices=["reorder", "natural", "auto", "stage1", "stage2"],
+                    help="which stages the plan of the timed step runs (Section 6.5 ablation); the headline is 'auto': "
+                         "the guard of Section 4.5 decides per head whether reordering pays")
     ap.add_argument("--mask", default="videomask", choices=["videomask", "random20", "dense"],
                     help="mask generator: the config's structured recipe, 20 %% uniform columns per row "
                          "(the paper's Random row), or all pairs (dense run for the gap metric)")

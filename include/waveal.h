@@ -101,8 +101,8 @@ typedef struct waveal_plan_out {
                            (an index list entry out of range); the caller zeroes it          */
 } waveal_plan_out;
 
-/* Fills `desc` with the library defaults (T = 5, AUTO, guard: K+V of a head within a quarter
- * of L2, density below 1 %, natural-order locality of at least 1/2);
+/* Fills `desc` with the library defaults (T = 5, AUTO, guard: K+V of a head within 9/16 of
+ * L2, density below 1 %, natural-order locality of at least 1/2);
  * heads / block counts stay 0 for the caller to set.  Host-only, no CUDA call. */
 void waveal_plan_desc_default(waveal_plan_desc* desc /*host*/);
 

@@ -245,7 +245,7 @@ def guard_stats(mask: np.ndarray, wave: int) -> Dict[str, int]:
             "pair2": int(((sizes - 1) * t).sum())}
 
 
-DEFAULT_GUARD = dict(kv_bytes_per_head=0, l2_bytes=0, l2_fit_num=1, l2_fit_den=4,
+DEFAULT_GUARD = dict(kv_bytes_per_head=0, l2_bytes=0, l2_fit_num=9, l2_fit_den=16,
                      min_density_ppm=10000, min_nnz=0, local_num=1, local_den=2)
 
 

@@ -43,7 +43,7 @@ constexpr int kProducerWarp = 0, kPvWarp = 1, kSoftmaxWarp0 = 2, kQkWarp = 10;
 constexpr long long kTimeoutCycles = 4000000000ll;   // ~2 s at boost clock
 constexpr long long kSelfTestCycles = 4000000ll;     // ~2 ms: wait limit under WAVEAL_ATTN_SELFTEST_LOST_TILE
 #ifndef WAVEAL_POLY_EVERY
-#define WAVEAL_POLY_EVERY 2
+#define WAVEAL_POLY_EVERY 4
 #endif
 constexpr int kPolyEvery = WAVEAL_POLY_EVERY;          // n > 0: 1 pair of elements in n takes 2^x from the FMA pipe (0 = all from the transcendental unit)
 
@@ -287,7 +287,7 @@ struct Geo {
   static constexpr int NKS = (NSTAGE + 1) / 2;       // K tile ring
   static constexpr int NVS = NSTAGE / 2;             // V tile ring
   static constexpr int NSBUF = 3;                    // S/P buffers in tensor memory
-  static constexpr int CH = BK < 64 ? BK : 64;       // S columns a softmax thread holds at a time
+  static constexpr int CH = 32;                      // S columns a softmax thread holds at a time
   static constexpr int NCH = BK / CH;                // such chunks per row
   static constexpr int CO = D / 2;                   // O columns per epilogue thread
   static constexpr int OFF_Q = 0;
@@ -790,7 +790,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           float ls4[4] = {0.f, 0.f, 0.f, 0.f};
           // ---- pass 2: exponentials; P_j (bf16 pairs) goes over the first half of the row's own
           // S columns, each chunk after its S values have been read
-#pragma unroll
+#pragma unroll 1
           for (int ch = 0; ch < G::NCH; ++ch) {
             uint32_t sv[G::CH];
 #pragma unroll
@@ -818,7 +818,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
             if constexpr (G::CH == 64) { WAVEAL_TMEM_ST32(s_addr + ch * 32, pk, 0); }
             else { WAVEAL_TMEM_ST16(s_addr + ch * 16, pk, 0); }
-            if (G::NCH == 2 && ch == 0) {
+            if (G::NCH >= 2 && ch == G::NCH / 2 - 1) {
               // first half of P_j: its MMAs can run while the second half is computed
               tc_wait_st();
               tc_fence_before();
@@ -837,7 +837,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           tc_fence_before();
           __syncwarp();
           if (lane == 0) {
-            if (G::NCH != 2) mbar_arrive(BAR(B_P_FULL + sb * 2));
+            if (G::NCH < 2) mbar_arrive(BAR(B_P_FULL + sb * 2));
             mbar_arrive(BAR(B_P_FULL + sb * 2 + 1));
           }
         }

@@ -660,7 +660,7 @@ extern "C" void waveal_plan_desc_default(waveal_plan_desc* d) {
   *d = waveal_plan_desc{};
   d->svd_iters = 5;    // low end of the paper's 5-15: the attention time did not move between 3, 5 and 10 on the measured shapes
   d->mode = WAVEAL_AUTO;
-  d->l2_fit_num = 1; d->l2_fit_den = 4;
+  d->l2_fit_num = 9; d->l2_fit_den = 16;   // calibrated on the B200 (calibrate_guard): no gain up to K+V = 0.57 x L2 on either mask family
   d->min_density_ppm = 10000;
   d->local_num = 1; d->local_den = 2;
   d->min_nnz = 0;

@@ -38,7 +38,7 @@ def test_struct_layouts():
 def test_defaults_and_workspace_query(lib):
     d = wb.plan_desc_default()
     assert (d.svd_iters, d.mode, d.l2_fit_num, d.l2_fit_den, d.min_density_ppm, d.local_num, d.local_den) == \
-        (5, wb.AUTO, 1, 4, 10000, 1, 2)
+        (5, wb.AUTO, 9, 16, 10000, 1, 2)
     with pytest.raises(wb.WavealError) as e:
         wb.plan_workspace_bytes(d)                       # heads etc. still 0
     assert e.value.status == wb.ERR_INVALID_ARG and "positive" in str(e.value)

@@ -112,9 +112,9 @@ def test_guard_decisions_per_head():
     sparse[0, :] = False
     sparse[0, 0] = True
     masks = [rnd, loc, sparse]
-    guard = dict(wo.DEFAULT_GUARD, kv_bytes_per_head=1000, l2_bytes=3000, min_density_ppm=20000)
+    guard = dict(wo.DEFAULT_GUARD, kv_bytes_per_head=2000, l2_bytes=3000, min_density_ppm=20000)
     d = wb.plan_desc_default(heads=3, n_q_blocks=m, n_kv_blocks=m, wave_size=8, mode=wb.AUTO, seed=3,
-                             kv_bytes_per_head=1000, l2_bytes=3000, min_density_ppm=20000)
+                             kv_bytes_per_head=2000, l2_bytes=3000, min_density_ppm=20000)
     res = wb.plan_bitmap(d, _bitmap_dev(masks), debug=True)
     torch.cuda.synchronize()
     flags = _np(res.skip_flags).tolist()

@@ -321,7 +321,9 @@ def test_guard_cases():
     # short sequence: the head's K+V fit the cache budget
     f = wo.guard_flags(mk, 8, {**g, "kv_bytes_per_head": 10, "l2_bytes": 100})
     assert f & wo.FLAG_SHORT_SEQ
-    f = wo.guard_flags(mk, 8, {**g, "kv_bytes_per_head": 26, "l2_bytes": 100})
+    f = wo.guard_flags(mk, 8, {**g, "kv_bytes_per_head": 56, "l2_bytes": 100})      # 56/100 <= 9/16
+    assert f & wo.FLAG_SHORT_SEQ
+    f = wo.guard_flags(mk, 8, {**g, "kv_bytes_per_head": 57, "l2_bytes": 100})
     assert not f & wo.FLAG_SHORT_SEQ
     # too sparse
     sparse = np.eye(200, dtype=bool)
