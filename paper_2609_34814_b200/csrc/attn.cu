@@ -8,23 +8,24 @@
 // SM, take tickets from a global counter, so a freed SM starts the next row of the list at
 // once - the streaming "wave" behaviour of Section 2.3 that the schedule is built for.
 //
-// Structure of one CTA (352 threads):
+// Structure of one CTA (608 threads):
 //   warp 0      producer: takes tickets, publishes tasks, issues TMA loads of the Q tile and
 //               of the K and V tiles (128-byte-swizzled slabs) into two shared-memory rings
-//   warp 10     MMA issuer 1: S_j = Q K_j^T (operands in shared memory) into one of three S
+//   warp 18     MMA issuer 1: S_j = Q K_j^T (operands in shared memory) into one of three S
 //               buffers in tensor memory, up to three blocks ahead of the softmax
 //   warp 1      MMA issuer 2: O += P_j V_j (P read from tensor memory, where it lies over the
 //               columns S_j came from), fp32 accumulator in tensor memory.  Two issuing warps:
 //               the waits and ring arithmetic of one run while the other's MMAs execute
-//   warps 2-9   softmax, two teams of four warps that take the KV blocks of a task in turn:
-//               a thread owns one row of S for its team's blocks (row max, then exponentials
-//               and P in a second read of S); on every scheduler one warp of each team is
-//               resident, half a block apart, so one team's waits and loads hide behind the
-//               other's arithmetic.  The teams hand each other the running reference max of
-//               every row through shared memory; each keeps the row sum of its own blocks;
-//               O in tensor memory is rescaled only when the max grew by more than 2^8; the
-//               epilogue adds the two sums, normalises and stores O at the ORIGINAL row (no
-//               inverse permutation)
+//   warps 2-17  softmax, two teams of eight warps that take the KV blocks of a task in turn;
+//               inside a team a row of S has two owners, one per half of its columns (row max
+//               in the blocks that take one, then exponentials and P in a second read of S,
+//               32 columns at a time in a rolled loop).  On every scheduler two warps of each
+//               team are resident, the teams half a block apart, so one team's waits and loads
+//               hide behind the other's arithmetic.  The teams hand each other the running
+//               reference max of every row through shared memory; every thread keeps the row
+//               sum of its own columns; O in tensor memory is rescaled only when the max grew
+//               by more than 2^8; the epilogue adds the four partial sums of a row, normalises
+//               and stores O at the ORIGINAL row (no inverse permutation)
 // Two launches per call: in the first the row max is taken in blocks 0 and 1 of a task only and
 // the reference stays fixed afterwards (softmax does not depend on it short of overflow); a task
 // in which a block's sum of exponentials reaches 2^24 is listed in the workspace and computed
@@ -38,8 +39,8 @@
 
 namespace {
 
-constexpr int kThreads = 352;
-constexpr int kProducerWarp = 0, kPvWarp = 1, kSoftmaxWarp0 = 2, kQkWarp = 10;
+constexpr int kThreads = 608;
+constexpr int kProducerWarp = 0, kPvWarp = 1, kSoftmaxWarp0 = 2, kQkWarp = 18;
 constexpr long long kTimeoutCycles = 4000000000ll;   // ~2 s at boost clock
 constexpr long long kSelfTestCycles = 4000000ll;     // ~2 ms: wait limit under WAVEAL_ATTN_SELFTEST_LOST_TILE
 #ifndef WAVEAL_POLY_EVERY
@@ -218,6 +219,20 @@ __device__ __forceinline__ void ex2_fma2(float& e0, float& e1, float s0, float s
       ::WAVEAL_IN32(v, o), "r"(taddr)                                                            \
       : "memory")
 
+// 16 consecutive fp32 columns
+#define WAVEAL_TMEM_LD16(taddr, v, o)                                                            \
+  asm volatile(                                                                                  \
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "                                                  \
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"           \
+      : "=r"(v[o+0]), "=r"(v[o+1]), "=r"(v[o+2]), "=r"(v[o+3]), "=r"(v[o+4]), "=r"(v[o+5]), "=r"(v[o+6]), "=r"(v[o+7]), \
+        "=r"(v[o+8]), "=r"(v[o+9]), "=r"(v[o+10]), "=r"(v[o+11]), "=r"(v[o+12]), "=r"(v[o+13]), "=r"(v[o+14]), "=r"(v[o+15]) \
+      : "r"(taddr)                                                                               \
+      : "memory")
+#define WAVEAL_TMEM_WAIT_LD16(v, o)                                                              \
+  asm volatile("tcgen05.wait::ld.sync.aligned;"                                                  \
+      : "+r"(v[o+0]), "+r"(v[o+1]), "+r"(v[o+2]), "+r"(v[o+3]), "+r"(v[o+4]), "+r"(v[o+5]), "+r"(v[o+6]), "+r"(v[o+7]), \
+        "+r"(v[o+8]), "+r"(v[o+9]), "+r"(v[o+10]), "+r"(v[o+11]), "+r"(v[o+12]), "+r"(v[o+13]), "+r"(v[o+14]), "+r"(v[o+15]) \
+      ::"memory")
 #define WAVEAL_TMEM_ST16(taddr, v, o)                                                            \
   asm volatile(                                                                                  \
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "                                           \
@@ -287,17 +302,18 @@ struct Geo {
   static constexpr int NKS = (NSTAGE + 1) / 2;       // K tile ring
   static constexpr int NVS = NSTAGE / 2;             // V tile ring
   static constexpr int NSBUF = 3;                    // S/P buffers in tensor memory
+  static constexpr int HC = BK / 2;                  // S columns of a row one softmax thread owns (a row has two owners)
   static constexpr int CH = 32;                      // S columns a softmax thread holds at a time
-  static constexpr int NCH = BK / CH;                // such chunks per row
-  static constexpr int CO = D / 2;                   // O columns per epilogue thread
+  static constexpr int NCH = HC / CH;                // such chunks per thread and block
+  static constexpr int CO = D / 4;                   // O columns per epilogue thread
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + Q_BYTES;
   static constexpr int OFF_V = OFF_K + NKS * TILE_BYTES;
   static constexpr int OFF_BAR = OFF_V + NVS * TILE_BYTES;
-  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 4 * NSBUF + 2 + 2 + 8 + 4;
+  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 4 * NSBUF + 2 + 2 + 8 + 4 + 8;
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
   static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
-  static constexpr int OFF_MISC = OFF_MX + 2 * 128 * 4 + 2 * 2 * 128 * 8;
+  static constexpr int OFF_MISC = OFF_MX + 4 * 128 * 4 + 2 * 2 * 2 * 128 * 4 + 2 * 4 * 128 * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;   // + slack for 1024-byte alignment
   // tensor memory: three S/P buffers of 128 columns, then the output accumulator
   static constexpr uint32_t S_STRIDE = 128, O_COL = 384, TMEM_COLS = 512;
@@ -361,11 +377,12 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 B_K_EMPTY = B_K_FULL + G::NKS, B_V_FULL = B_K_EMPTY + G::NKS, B_V_EMPTY = B_V_FULL + G::NVS,
                 B_S_FULL = B_V_EMPTY + G::NVS, B_P_FULL = B_S_FULL + G::NSBUF, B_S_FREE = B_P_FULL + 2 * G::NSBUF,
                 B_O_FULL = B_S_FREE + G::NSBUF, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1, B_MX = B_FINAL + 2,
-                B_EX = B_MX + 8;
-  static_assert(B_EX + 4 <= G::N_BAR, "barrier count");
+                B_EX = B_MX + 8, B_HX = B_EX + 4;
+  static_assert(B_HX + 8 <= G::N_BAR, "barrier count");
   Task* tasks = reinterpret_cast<Task*>(smem + G::OFF_TASK);
-  volatile float* mpub = reinterpret_cast<volatile float*>(smem + G::OFF_MX);   // [block parity][128] reference max after a block
-  float2* ex = reinterpret_cast<float2*>(smem + G::OFF_MX + 2 * 128 * 4);       // [task parity][team][128] (reference, sum)
+  volatile float* mpub = reinterpret_cast<volatile float*>(smem + G::OFF_MX);   // [block index mod 4][128] reference max after a block
+  volatile float* mhalf = reinterpret_cast<volatile float*>(smem + G::OFF_MX + 4 * 128 * 4);   // [use parity][team][column half][128] max of a half row
+  float2* ex = reinterpret_cast<float2*>(smem + G::OFF_MX + 4 * 128 * 4 + 2 * 2 * 2 * 128 * 4);    // [task parity][team*2+half][128] (reference, sum)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + G::OFF_MISC);
   volatile int* abort_smem = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 4);
   volatile int* redo_flag = reinterpret_cast<volatile int*>(smem + G::OFF_MISC + 8);   // [task parity]
@@ -373,24 +390,25 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const long long t_start = clock64();
 
   if (tid == 0) {
-    // a task is read by the two MMA issuers and the eight softmax warps
-    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_TASK_FULL + i), 1); mbar_init(BAR(B_TASK_EMPTY + i), 10); }
+    // a task is read by the two MMA issuers and the sixteen softmax warps
+    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_TASK_FULL + i), 1); mbar_init(BAR(B_TASK_EMPTY + i), 18); }
     mbar_init(BAR(B_Q_FULL), 1);
     mbar_init(BAR(B_Q_EMPTY), 1);
     for (int i = 0; i < G::NKS; ++i) { mbar_init(BAR(B_K_FULL + i), 1); mbar_init(BAR(B_K_EMPTY + i), 1); }
     for (int i = 0; i < G::NVS; ++i) { mbar_init(BAR(B_V_FULL + i), 1); mbar_init(BAR(B_V_EMPTY + i), 1); }
     for (int i = 0; i < G::NSBUF; ++i) {
       mbar_init(BAR(B_S_FULL + i), 1);
-      mbar_init(BAR(B_P_FULL + 2 * i), 4);      // one per half of P (the four warps of the owning team)
+      mbar_init(BAR(B_P_FULL + 2 * i), 4);      // one per half of P (the four warps that own that half in the block's team)
       mbar_init(BAR(B_P_FULL + 2 * i + 1), 4);
       mbar_init(BAR(B_S_FREE + i), 1);
     }
     mbar_init(BAR(B_O_FULL), 1);
-    mbar_init(BAR(B_O_FREE), 8);
+    mbar_init(BAR(B_O_FREE), 16);
     mbar_init(BAR(B_FINAL), 1);
     mbar_init(BAR(B_FINAL + 1), 1);
     for (int i = 0; i < 8; ++i) mbar_init(BAR(B_MX + i), 1);
-    for (int i = 0; i < 4; ++i) mbar_init(BAR(B_EX + i), 2);    // the two warps of a lane quadrant, once per task
+    for (int i = 0; i < 4; ++i) mbar_init(BAR(B_EX + i), 4);    // the four warps of a lane quadrant, once per task
+    for (int i = 0; i < 8; ++i) mbar_init(BAR(B_HX + i), 2);    // the two owners of a row (team, quadrant), once per max
     *abort_smem = 0;
     redo_flag[0] = 0;
     redo_flag[1] = 0;
@@ -632,7 +650,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #pragma unroll
           for (int kk = 0; kk < G::BK / 32; ++kk) {
             const int k = h * (G::BK / 32) + kk;
-            umma_bf16_ts(d_o, pbase + k * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+            // P of key half h lies over the first columns of that half's own S columns
+            umma_bf16_ts(d_o, pbase + h * G::HC + kk * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
           }
         }
         if (!ok) break;
@@ -655,22 +674,26 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
   } else {
     // ============================================================== softmax / epilogue
-    // Two teams of four warps take the KV blocks of a task in turn (team = block index mod 2);
-    // a thread owns one whole row of S for its team's blocks.  On every scheduler sits one warp
-    // of each team, half a block apart in time: while one is in its exponentials (bound by the
-    // transcendental unit) the other waits for S, loads it, takes the row max and stores P, so
-    // the latencies of one team hide behind the arithmetic of the other.  Nothing is exchanged
-    // inside a row; the teams only hand the running reference max of each row to each other
-    // (shared memory + one mbarrier per lane quadrant and block parity), because both
-    // accumulate into the same O.  Each team keeps the sum of its own blocks; the epilogue adds
-    // the two.
-    const int sw = warp - kSoftmaxWarp0;       // 0..7
+    // Sixteen warps: two teams take the KV blocks of a task in turn (team = block index mod 2),
+    // and inside a team a row of S has two owners, one per half of its columns (a warp can reach
+    // only the 32 tensor-memory lanes of its quadrant, so the two owners of a row sit in warps
+    // four apart).  Four softmax warps per scheduler instead of two: the loop is bound by
+    // instruction issue and latency, and twice the warps hide twice the latency.  The owners
+    // of a row share its reference max (exchanged through shared memory in the blocks that
+    // take one); each keeps the sum of its own columns; P of a column half is written over the
+    // first columns of that half's own S columns and released with its own barrier.  The two
+    // teams hand each other the running reference of each row (shared memory + one mbarrier
+    // per lane quadrant and block parity), because both accumulate into the same O.  The
+    // epilogue adds the four partial sums of a row.
+    const int sw = warp - kSoftmaxWarp0;       // 0..15
     const int quad = warp & 3;                 // tensor-memory lane quadrant this warp may access
-    const int team = sw >> 2;                  // owns blocks j with (j & 1) == team; epilogue: half of the O columns
+    const int team = (sw >> 2) & 1;            // owns blocks j with (j & 1) == team
+    const int half = sw >> 3;                  // column half of S; epilogue: quarter team*2+half of the O columns
     const int r = quad * 32 + lane;            // row of the 128-row MMA tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t o_row = tmem_base + lane_addr + G::O_COL;
-    uint32_t task_it = 0, s_phase = 0, o_it = 0, mx_phase = 0, sb = 0;   // s_phase bit b: parity of the uses of S[b] so far
+    const int part = team * 2 + half;
+    uint32_t task_it = 0, s_phase = 0, o_it = 0, mx_phase = 0, hx_it = 0, sb = 0;   // s_phase bit b: parity of the uses of S[b] so far
     bool ok = true;
     while (ok) {
       const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
@@ -679,22 +702,22 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const Task tk = tasks[slot];
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + slot));
-      float2* exb = ex + (task_it & 1) * 256;
+      float2* exb = ex + (task_it & 1) * 512;
       const uint32_t rslot = task_it & 1;
       ++task_it;
       if (tk.n < 0) break;
       const long long q_tok = (long long)tk.row * G::BQ + r;
       const bool row_live = r < G::BQ && q_tok < p.seq_q;
-      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + team * G::CO;
+      __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + part * G::CO;
       if (tk.n == 0) {
         if (row_live) {
 #pragma unroll
           for (int c = 0; c < G::CO / 8; ++c) reinterpret_cast<uint4*>(o_ptr)[c] = make_uint4(0, 0, 0, 0);
-          if (p.lse && team == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
+          if (p.lse && part == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = -INFINITY;
         }
         continue;
       }
-      // l_run: sum over this team's blocks, relative to the reference m_ref
+      // l_run: sum over this thread's columns of this team's blocks, relative to the reference m_ref
       float m_ref = -INFINITY, l_run = 0.f;
       for (int j = 0; j < tk.n && ok; ++j) {
         const uint32_t par = (uint32_t)j & 1u;
@@ -702,10 +725,11 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           ok = warp_wait(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE;
+          const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE + half * G::HC;
           const bool ragged = j == tk.n - 1 && tk.tail_valid < G::BK;
+          const int col0 = half * G::HC;       // first key of the block this thread looks at
           // ---- pass 1: row max (the values are loaded again for the exponentials: a second
-          // tensor-memory load is cheaper than 128 live registers)
+          // tensor-memory load is cheaper than keeping them in registers)
           // In the first pass over the tasks (FAST) only blocks 0 and 1 of a task take a max and
           // may move the reference; from block 2 on both teams keep the reference of block 1.
           // Any reference gives the same softmax as long as nothing overflows, so the later
@@ -714,30 +738,39 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           // max of every block (the rule of the paper's online softmax).
           const bool fixed_ref = FAST && j >= 2;
           float mloc = -INFINITY;
-          if (!fixed_ref)
+          if (!fixed_ref) {
+#pragma unroll 1
+            for (int ch = 0; ch < G::NCH; ++ch) {
+              uint32_t sv[G::CH];
+              WAVEAL_TMEM_LD32(s_addr + ch * G::CH, sv, 0);
+              WAVEAL_TMEM_WAIT_LD32(sv, 0);
+              // scores of keys beyond seq_kv (ragged last block) do not exist
+              if (ragged) {
 #pragma unroll
-          for (int ch = 0; ch < G::NCH; ++ch) {
-            uint32_t sv[G::CH];
+                for (int c = 0; c < G::CH; ++c)
+                  if (col0 + ch * G::CH + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
+              }
+              float mx8[8];
 #pragma unroll
-            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_LD32(s_addr + ch * G::CH + c, sv, c);
+              for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(sv[i]);
 #pragma unroll
-            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_WAIT_LD32(sv, c);
-            // scores of keys beyond seq_kv (ragged last block) do not exist
-            if (ragged) {
+              for (int c = 8; c < G::CH; c += 8) {
 #pragma unroll
-              for (int c = 0; c < G::CH; ++c)
-                if (ch * G::CH + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
+                for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(sv[c + i]));
+              }
+              mloc = fmaxf(mloc, fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                                       fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7]))));
             }
-            float mx8[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) mx8[i] = __uint_as_float(sv[i]);
-#pragma unroll
-            for (int c = 8; c < G::CH; c += 8) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) mx8[i] = fmaxf(mx8[i], __uint_as_float(sv[c + i]));
-            }
-            mloc = fmaxf(mloc, fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                                     fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7]))));
+            // the other owner of the row (same team and quadrant, other column half)
+            // (two buffers by use parity: the partner's next value cannot land on one not yet read)
+            volatile float* mh = mhalf + (hx_it & 1u) * 512;
+            mh[(team * 2 + half) * 128 + r] = mloc;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR(B_HX + team * 4 + quad));
+            ok = warp_wait(ctx, BAR(B_HX + team * 4 + quad), hx_it & 1u, 26);
+            if (!ok) break;
+            ++hx_it;
+            mloc = fmaxf(mloc, mh[(team * 2 + (half ^ 1)) * 128 + r]);
           }
           // ---- the row's reference after block j-1, from the other team
           float m_prev = m_ref;
@@ -745,15 +778,18 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             // that team's arrival for block j-1 is phase number (arrivals of that parity so far) - 1
             ok = warp_wait(ctx, BAR(B_MX + quad * 2 + (par ^ 1u)), ((mx_phase >> (par ^ 1u)) & 1u) ^ 1u, 24);
             if (!ok) break;
-            m_prev = mpub[(par ^ 1u) * 128 + r];
+            m_prev = mpub[((j - 1) & 3) * 128 + r];
           }
           const float m_cand = fmaxf(m_prev, mloc * p.sl2);
           // keep the stale reference unless it is exceeded by more than 2^8 (exact: the final
-          // normalisation divides by a sum taken with the same reference)
+          // normalisation divides by a sum taken with the same reference); both owners of a row
+          // see the same values and take the same decision
           const bool grow = !fixed_ref && __any_sync(0xffffffffu, m_cand > m_prev + 8.0f);
           const float m_new = grow ? m_cand : m_prev;
-          if (!fixed_ref) {
-            mpub[par * 128 + r] = m_new;
+          if (!fixed_ref && half == 0) {
+            // (slot j mod 4: the owner of block j+4 cannot get there before both owners of block
+            // j+1 have read this one)
+            mpub[(j & 3) * 128 + r] = m_new;
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR(B_MX + quad * 2 + par));
           }
@@ -764,15 +800,16 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           // rare: the reference grew, so O (blocks 0..j-1) is rescaled; its last MMA (block j-1)
           // must be complete: that is the latest phase of the barrier of the S buffer before
           // this one (the next P V on that buffer needs a P this team has not produced yet).
-          // Done before any part of P_j is released to the MMA warp.
+          // Done before any part of P_j is released to the MMA warp; each owner takes half of
+          // the row's output columns.
           if (grow && j > 0) {
             const uint32_t sbp = sb == 0 ? (uint32_t)G::NSBUF - 1u : sb - 1u;
             ok = warp_wait(ctx, BAR(B_S_FREE + sbp), ((s_phase >> sbp) & 1u) ^ 1u, 22);
             if (!ok) break;
             tc_fence_after();
             const float alpha = ex2(m_prev - m_new);
-#pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
+#pragma unroll 1
+            for (int c0 = half * (D / 2); c0 < (half + 1) * (D / 2); c0 += 32) {
               uint32_t ov[32];
               WAVEAL_TMEM_LD32(o_row + c0, ov, 0);
               WAVEAL_TMEM_WAIT_LD32(ov, 0);
@@ -788,19 +825,18 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           const float neg_m = ((m_new == -INFINITY) ? 0.f : -m_new) + 0.0028150156f;
           const float a128 = p.sl2 * 0.0078125f, b128 = (neg_m - kPolyLo) * 0.0078125f;   // polynomial share
           float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-          // ---- pass 2: exponentials; P_j (bf16 pairs) goes over the first half of the row's own
-          // S columns, each chunk after its S values have been read
+          // ---- pass 2: exponentials; P (bf16 pairs) goes over the first half of the thread's own
+          // S columns, each chunk after its S values have been read.  A rolled loop over
+          // 32-column chunks: the body stays small enough for the instruction cache.
 #pragma unroll 1
           for (int ch = 0; ch < G::NCH; ++ch) {
             uint32_t sv[G::CH];
-#pragma unroll
-            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_LD32(s_addr + ch * G::CH + c, sv, c);
-#pragma unroll
-            for (int c = 0; c < G::CH; c += 32) WAVEAL_TMEM_WAIT_LD32(sv, c);
+            WAVEAL_TMEM_LD32(s_addr + ch * G::CH, sv, 0);
+            WAVEAL_TMEM_WAIT_LD32(sv, 0);
             if (ragged) {
 #pragma unroll
               for (int c = 0; c < G::CH; ++c)
-                if (ch * G::CH + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
+                if (col0 + ch * G::CH + c >= tk.tail_valid) sv[c] = __float_as_uint(-INFINITY);
             }
             uint32_t pk[G::CH / 2];
 #pragma unroll
@@ -816,30 +852,19 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
               fadd2(ls4[c & 2], ls4[(c & 2) + 1], ls4[c & 2], ls4[(c & 2) + 1], e0, e1);
               pk[c / 2] = __byte_perm(__float_as_uint(e0), __float_as_uint(e1), 0x7632);
             }
-            if constexpr (G::CH == 64) { WAVEAL_TMEM_ST32(s_addr + ch * 32, pk, 0); }
-            else { WAVEAL_TMEM_ST16(s_addr + ch * 16, pk, 0); }
-            if (G::NCH >= 2 && ch == G::NCH / 2 - 1) {
-              // first half of P_j: its MMAs can run while the second half is computed
-              tc_wait_st();
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb * 2));
-            }
+            WAVEAL_TMEM_ST16(s_addr + ch * 16, pk, 0);
           }
           const float l_blk = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
           l_run += l_blk;
           // all terms are positive (the transcendental unit returns +inf on overflow, the
-          // polynomial share saturates at 2^28), so a block sum below 2^24 bounds every exponent
-          // of the block; at or above it (or not a number) the fixed reference is too far off:
+          // polynomial share saturates at 2^28), so a sum below 2^24 bounds every exponent it
+          // covers; at or above it (or not a number) the fixed reference is too far off:
           // redo the task
           if (fixed_ref && __any_sync(0xffffffffu, !(l_blk < kRedoLimit))) redo_flag[rslot] = 1;
           tc_wait_st();
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) {
-            if (G::NCH < 2) mbar_arrive(BAR(B_P_FULL + sb * 2));
-            mbar_arrive(BAR(B_P_FULL + sb * 2 + 1));
-          }
+          if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb * 2 + half));
         }
         // both teams count every block
         s_phase ^= 1u << sb;
@@ -847,8 +872,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
       if (!ok) break;
-      // ---- epilogue: O / l at the original row position; l = the two teams' sums brought to
-      // the final reference (the larger of the two, references never shrink)
+      // ---- epilogue: O / l at the original row position; l = the four partial sums of the row
+      // brought to the final reference (the larger of the two teams', references never shrink)
       ok = warp_wait(ctx, BAR(B_O_FULL), o_it & 1, 23);
       if (!ok) break;
       ++o_it;
@@ -861,24 +886,24 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         p.ws[9 + 2 * e] = tk.row;
         redo_flag[rslot] = 0;
       }
-      exb[team * 128 + r] = make_float2(m_ref, l_run);
-      // the partner warp of this lane quadrant (other team) has written its half: a bounded wait
-      // like every other, so that a warp whose partner gave up does not stay behind
+      exb[part * 128 + r] = make_float2(m_ref, l_run);
+      // the other three warps of this lane quadrant have written their parts: a bounded wait
+      // like every other, so that a warp whose partners gave up does not stay behind
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_EX + quad));
       ok = warp_wait(ctx, BAR(B_EX + quad), (o_it & 1) ^ 1, 25);
       if (!ok) break;
-      const float2 oth = exb[(team ^ 1) * 128 + r];
-      const float m_all = fmaxf(m_ref, oth.x);
-      const float a_self = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_all);
-      const float a_oth = (oth.x == -INFINITY) ? 0.f : ex2(oth.x - m_all);
-      const float l_tot = a_self * l_run + a_oth * oth.y;
+      const float2 e00 = exb[0 * 128 + r], e01 = exb[1 * 128 + r], e10 = exb[2 * 128 + r], e11 = exb[3 * 128 + r];
+      const float m0 = fmaxf(e00.x, e01.x), m1 = fmaxf(e10.x, e11.x);     // the two owners of a team agree; a team
+      const float m_all = fmaxf(m0, m1);                                   // without blocks (n == 1) has -inf
+      const float a0 = (m0 == -INFINITY) ? 0.f : ex2(m0 - m_all);
+      const float a1 = (m1 == -INFINITY) ? 0.f : ex2(m1 - m_all);
+      const float l_tot = a0 * (e00.y + e01.y) + a1 * (e10.y + e11.y);
       const float inv_l = 1.0019531f / l_tot;    // the sums carry the centring factor 1 + 2^-9
       uint32_t ov[G::CO];
-#pragma unroll
-      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_LD32(o_row + team * G::CO + c, ov, c);
-#pragma unroll
-      for (int c = 0; c < G::CO; c += 32) WAVEAL_TMEM_WAIT_LD32(ov, c);
+      static_assert(G::CO == 32 || G::CO == 16, "a quarter of head_dim 128 or 64");
+      if constexpr (G::CO == 32) { WAVEAL_TMEM_LD32(o_row + part * G::CO, ov, 0); WAVEAL_TMEM_WAIT_LD32(ov, 0); }
+      else { WAVEAL_TMEM_LD16(o_row + part * G::CO, ov, 0); WAVEAL_TMEM_WAIT_LD16(ov, 0); }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_O_FREE));
@@ -894,7 +919,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           }
           *reinterpret_cast<uint4*>(o_ptr + c) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (p.lse && team == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_all + log2f(l_tot) - 0.0028150156f) * 0.6931471805599453f;
+        if (p.lse && part == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_all + log2f(l_tot) - 0.0028150156f) * 0.6931471805599453f;
       }
     }
   }
