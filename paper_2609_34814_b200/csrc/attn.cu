@@ -268,7 +268,22 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 
 // ------------------------------------------------------------------ kernel
 
-struct Task { int h, row, lo, n, tail_valid, pad0, pad1, pad2; };
+// n: KV tiles of the task (a tile = 128 keys = 128/block consecutive entries of the row's list),
+// len: entries of the list, tail_valid: keys of the last tile that exist
+struct Task { int h, row, lo, n, tail_valid, len, pad1, pad2; };
+
+// tiles, list length and valid keys of the last tile from a list of `len` blocks of `block` keys
+// whose last entry is `last`
+__host__ __device__ inline void fill_tiles(Task& tk, int len, int block, int last, int n_b, int seq_kv) {
+  const int kb = 128 / block;
+  tk.len = len;
+  tk.n = (len + kb - 1) / kb;
+  tk.tail_valid = 128;
+  if (len > 0) {
+    tk.tail_valid = (len - (tk.n - 1) * kb) * block;
+    if ((seq_kv % block) != 0 && last == n_b - 1) tk.tail_valid -= block - seq_kv % block;
+  }
+}
 
 struct AttnParams {
   __nv_bfloat16* O;
@@ -292,7 +307,11 @@ struct AttnParams {
 
 template <int BLOCK, int D>
 struct Geo {
-  static constexpr int BQ = BLOCK, BK = BLOCK;
+  // A KV tile is always 128 keys wide: one 128-key block, or two 64-key blocks that follow each
+  // other in the row's list (their rows land one after the other in the tile, so the MMAs, the
+  // softmax and the rings see the same shapes for both block sizes; a list of odd length ends
+  // in a half tile whose missing keys are treated like keys beyond the sequence end)
+  static constexpr int BQ = BLOCK, BK = 128, KB = 128 / BLOCK;
   static constexpr int SLABS = D / 64;               // 128-byte column slabs of a Q/K/V tile
   static constexpr int Q_BYTES = SLABS * 128 * 128;  // smem reserved for the 128 MMA rows
   static constexpr int TILE_BYTES = SLABS * BK * 128;
@@ -454,15 +473,14 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         // one 32-byte load behind the ticket instead of a chain through three lists
         const uint4* e = reinterpret_cast<const uint4*>(p.table + t);
         const uint4 a = e[0], b = e[1];
-        tk.h = (int)a.x; tk.row = (int)a.y; tk.lo = (int)a.z; tk.n = (int)a.w; tk.tail_valid = (int)b.x;
+        tk.h = (int)a.x; tk.row = (int)a.y; tk.lo = (int)a.z; tk.n = (int)a.w; tk.tail_valid = (int)b.x; tk.len = (int)b.y;
       } else {
         int h = p.ws[8 + 2 * t], row = p.ws[9 + 2 * t];
         if (h < 0 || h >= p.heads) h = 0;
         if (row < 0 || row >= p.m_b) row = 0;
         int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
-        tk.h = h; tk.row = row; tk.lo = lo; tk.n = max(hi - lo, 0);
-        tk.tail_valid = G::BK;
-        if (tk.n > 0 && (p.seq_kv % G::BK) != 0 && p.kv_idx[hi - 1] == p.n_b - 1) tk.tail_valid = p.seq_kv % G::BK;
+        tk.h = h; tk.row = row; tk.lo = lo;
+        fill_tiles(tk, max(hi - lo, 0), BLOCK, hi > lo ? p.kv_idx[hi - 1] : 0, p.n_b, p.seq_kv);
       }
       const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
       ok = warp_wait(ctx, BAR(B_TASK_EMPTY + slot), ph ^ 1, 1);
@@ -486,20 +504,32 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       q_armed = true; q_armed_parity = q_it & 1;
       ++q_it;
       // K tiles run three blocks ahead of the V tiles, like the MMAs that consume them
-      int chunk_base = -64, my_idx = 0;
-      auto load_tile = [&](bool is_k, int j) -> bool {
-        if (j < chunk_base || j >= chunk_base + 32) {
-          chunk_base = j & ~31;
-          const int q = chunk_base + lane;
-          my_idx = q < tk.n ? p.kv_idx[tk.lo + q] : 0;
+      // entry q of the row's list (32 entries are fetched at a time, one per lane).  The K and the V
+      // stream of a task walk the list a few entries apart, so each has its own 32 entries:
+      // one shared set would be fetched again and again while the two sit on either side of
+      // a multiple of 32
+      int chunk_base[2] = {-64, -64}, my_idx[2] = {0, 0};
+      auto entry = [&](int q, int w) -> int {
+        if (q < chunk_base[w] || q >= chunk_base[w] + 32) {
+          chunk_base[w] = q & ~31;
+          const int e = chunk_base[w] + lane;
+          my_idx[w] = e < tk.len ? p.kv_idx[tk.lo + e] : 0;
         }
-        int blk = __shfl_sync(0xffffffffu, my_idx, j - chunk_base);
+        int blk = __shfl_sync(0xffffffffu, my_idx[w], q - chunk_base[w]);
         if (blk < 0 || blk >= p.n_b) {                   // malformed list: report it and stay in range
           if (lane == 0 && p.dev_status && atomicCAS(p.dev_status, 0, WAVEAL_ERR_BAD_MASK) == 0) {
             p.dev_status[1] = 30; p.dev_status[2] = tk.h; p.dev_status[3] = blk;
           }
           blk = 0;
         }
+        return blk;
+      };
+      auto load_tile = [&](bool is_k, int j) -> bool {
+        // the blocks of tile j: entries KB*j .. of the list (the last tile of an odd list has one)
+        const int nblk = G::KB == 1 ? 1 : min(G::KB, tk.len - G::KB * j);
+        int blk[G::KB];
+#pragma unroll
+        for (int e = 0; e < G::KB; ++e) blk[e] = e < nblk ? entry(G::KB * j + e, is_k ? 0 : 1) : 0;
         const uint32_t it = is_k ? k_it : v_it;
         const uint32_t nst = is_k ? (uint32_t)G::NKS : (uint32_t)G::NVS;
         const uint32_t st = it % nst, sph = (it / nst) & 1;
@@ -507,13 +537,18 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (!warp_wait(ctx, BAR(b_empty), sph ^ 1, 3)) return false;
         // (self-test of the abort path: one tile is never requested, so its consumer's wait runs out)
         const bool dropped = p.drop_tile && is_k && t == 0 && j == 0;
-        if (lane == 0 && !dropped) {
-          mbar_expect_tx(BAR(b_full), G::TILE_BYTES);
+        if (!dropped) {
+          // one lane per box: lane e*SLABS + s requests slab s of block e
+          if (lane == 0) mbar_expect_tx(BAR(b_full), (uint32_t)nblk * G::SLABS * BLOCK * 128);
+          __syncwarp();
           const CUtensorMap* tm = is_k ? &tmK : &tmV;
           const uint32_t dst = sbase + (is_k ? G::OFF_K : G::OFF_V) + st * G::TILE_BYTES;
+          const int e = lane / G::SLABS, sl = lane % G::SLABS;
+          int my_blk = blk[0];
 #pragma unroll
-          for (int s = 0; s < G::SLABS; ++s)
-            tma_load_3d(dst + s * G::KV_SLAB_BYTES, tm, s * 64, blk * G::BK, tk.h, BAR(b_full));
+          for (int i = 1; i < G::KB; ++i) if (e == i) my_blk = blk[i];
+          if (e < nblk)
+            tma_load_3d(dst + sl * G::KV_SLAB_BYTES + e * BLOCK * 128, tm, sl * 64, my_blk * BLOCK, tk.h, BAR(b_full));
         }
         if (dropped) { ++k_it; return true; }
         if (is_k) { k_armed |= 1u << st; k_parity = (k_parity & ~(1u << st)) | (sph << st); ++k_it; }
@@ -617,6 +652,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       ok = warp_wait(ctx, BAR(B_TASK_FULL + task_slot), task_ph, 10);
       if (!ok) break;
       const int n = __shfl_sync(0xffffffffu, tasks[task_slot].n, 0);
+      const bool half_tail = __shfl_sync(0xffffffffu, tasks[task_slot].tail_valid, 0) <= 64;
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + task_slot));
       task_slot ^= 1;
@@ -645,6 +681,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             if (!ok) break;
           }
           tc_fence_after();
+          // (the second half of a half tile has no keys: its V rows were never loaded)
+          if (G::KB == 2 && h == 1 && j == n - 1 && half_tail) continue;
           // V tile as the N x K operand with N (head_dim) contiguous: 8 keys per 1024-byte
           // group along K (16 keys = 2048 bytes per MMA), next 64 columns of head_dim one slab further
 #pragma unroll
@@ -965,13 +1003,13 @@ __global__ void k_task_table(AttnParams p, int block_k, Task* table) {
   const int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
   if (lo < 0 || hi < lo || (long long)hi > nnz) { report(32, lo < 0 ? lo : hi); bad = true; }
   Task tk{};
-  tk.h = h; tk.row = row; tk.lo = bad ? 0 : lo; tk.n = bad ? 0 : hi - lo;
-  tk.tail_valid = block_k;
-  if (tk.n > 0) {
-    const int last = p.kv_idx[hi - 1];
-    if (last < 0 || last >= p.n_b) { report(33, last); tk.n = 0; }
-    else if ((p.seq_kv % block_k) != 0 && last == p.n_b - 1) tk.tail_valid = p.seq_kv % block_k;
+  tk.h = h; tk.row = row; tk.lo = bad ? 0 : lo;
+  int len = bad ? 0 : hi - lo, last = 0;
+  if (len > 0) {
+    last = p.kv_idx[hi - 1];
+    if (last < 0 || last >= p.n_b) { report(33, last); len = 0; }
   }
+  fill_tiles(tk, len, block_k, last, p.n_b, p.seq_kv);
   table[t] = tk;
 }
 
