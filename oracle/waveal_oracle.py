@@ -197,6 +197,24 @@ def stage1_order(angles: np.ndarray) -> np.ndarray:
     return np.argsort(angles, kind="stable").astype(np.int64)
 
 
+def cut_ring_at_largest_gap(order1: np.ndarray, angles: np.ndarray) -> np.ndarray:
+    """Variant of Stage 1 (not in the paper's Algorithm 2; Section 4.3.1 says the polar angle
+    'unrolls the ring' of rows into a sequence but not where the ring is opened - Eq. 4's atan2
+    opens it at -pi, wherever that falls).  Here the ring is opened where two neighbouring rows
+    are farthest apart in angle: gaps of the sorted angles, the wrap-around gap
+    angle[first] + 2 pi - angle[last] included; the first of equal largest gaps wins; the row
+    behind the gap becomes the first of the sequence.  The result is a rotation of order1."""
+    m = len(order1)
+    if m < 2:
+        return order1.copy()
+    a = angles[order1]
+    gaps = np.empty(m)
+    gaps[:m - 1] = a[1:] - a[:-1]
+    gaps[m - 1] = (a[0] + 2.0 * math.pi) - a[m - 1]
+    k = int(np.argmax(gaps))               # first maximum
+    return np.concatenate([order1[k + 1:], order1[:k + 1]])
+
+
 def stage2_order(order1: np.ndarray, nnz: np.ndarray, wave: int) -> np.ndarray:
     """Algorithm 2, Stage 2: consecutive buckets of at most `wave` rows of order1; inside a
     bucket, descending block count, ties keeping their Stage-1 order; concatenate."""
@@ -270,10 +288,12 @@ def guard_flags(mask: np.ndarray, wave: int, g: Dict[str, int]) -> int:
 
 
 def plan_head(mask: np.ndarray, wave: int, iters: int, seed: int, head: int,
-              mode: int = MODE_AUTO, guard: Optional[Dict[str, int]] = None) -> Dict[str, np.ndarray]:
+              mode: int = MODE_AUTO, guard: Optional[Dict[str, int]] = None,
+              ring_cut: bool = False) -> Dict[str, np.ndarray]:
     """Algorithm 2 for one head, with the guard of Section 4.5 in front.
     Returns row_order (index list: position -> original row), order1 (Stage-1 order),
-    row_nnz, col_count, u, angles and flags."""
+    row_nnz, col_count, u, angles and flags.  ring_cut=True opens the angular ring at its
+    largest gap instead of at -pi (cut_ring_at_largest_gap; a variant, off by default)."""
     g = dict(DEFAULT_GUARD)
     if guard:
         g.update(guard)
@@ -295,6 +315,8 @@ def plan_head(mask: np.ndarray, wave: int, iters: int, seed: int, head: int,
         u = mfcsi(mask, iters, start_block(seed, head, m_b))
         ang = polar_angles(u)
         order1 = stage1_order(ang)
+        if ring_cut:
+            order1 = cut_ring_at_largest_gap(order1, ang)
     order = order1 if mode == MODE_STAGE1_ONLY else stage2_order(order1, nnz, wave)
     res.update(row_order=order, order1=order1, flags=flags, u=u, angles=ang)
     return res

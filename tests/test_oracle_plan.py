@@ -1,5 +1,6 @@
 """Pins for the reordering part of the CPU oracle (no GPU)."""
 import itertools
+import math
 import os
 
 import numpy as np
@@ -370,3 +371,73 @@ def test_gather_scatter_blocks_are_inverse_and_match_loops():
     for p in range(6):
         assert np.array_equal(g[p * 4:(p + 1) * 4], x[order[p] * 4:(order[p] + 1) * 4])
     assert np.array_equal(wo.scatter_blocks(g, order, 4), x)
+
+
+def test_ring_cut_by_hand_and_is_a_rotation():
+    # sorted angles -3.0, -2.9, 0.1, 0.2, 3.0: gaps 0.1, 3.0, 0.1, 2.8 and 0.283 around the back
+    ang = np.array([-3.0, -2.9, 0.1, 0.2, 3.0])
+    o1 = wo.stage1_order(ang)
+    assert o1.tolist() == [0, 1, 2, 3, 4]
+    assert wo.cut_ring_at_largest_gap(o1, ang).tolist() == [2, 3, 4, 0, 1]
+    # the wrap-around gap is the largest: nothing moves
+    ang = np.array([0.5, -0.5, 0.0, 1.0])
+    o1 = wo.stage1_order(ang)
+    assert wo.cut_ring_at_largest_gap(o1, ang).tolist() == o1.tolist() == [1, 2, 0, 3]
+    # equal largest gaps: the first one in sorted order
+    ang = np.array([-2.0, -1.0, 0.0, 1.0])      # gaps 1, 1, 1 and 2 pi - 3 = 3.28 around the back
+    assert wo.cut_ring_at_largest_gap(wo.stage1_order(ang), ang).tolist() == [0, 1, 2, 3]
+    ang = np.array([-3.0, -1.0, 1.0, 3.0])      # gaps 2, 2, 2, 0.283: the first 2
+    assert wo.cut_ring_at_largest_gap(wo.stage1_order(ang), ang).tolist() == [1, 2, 3, 0]
+    # all angles equal (degenerate embedding): natural order stays
+    z = np.zeros(7)
+    assert wo.cut_ring_at_largest_gap(wo.stage1_order(z), z).tolist() == list(range(7))
+    # random: a rotation of the Stage-1 order, and first/last are the two rows across the largest circular gap
+    rng = np.random.default_rng(4)
+    ang = rng.uniform(-math.pi, math.pi, 41)
+    o1 = wo.stage1_order(ang)
+    oc = wo.cut_ring_at_largest_gap(o1, ang)
+    doubled = np.concatenate([o1, o1]).tolist()
+    assert any(doubled[i:i + 41] == oc.tolist() for i in range(41))
+    circ = lambda a, b: (ang[b] - ang[a]) % (2 * math.pi)        # going up from a to b around the ring
+    best = max(circ(o1[i], o1[(i + 1) % 41]) for i in range(41))
+    assert abs(circ(oc[-1], oc[0]) - best) < 1e-12
+
+
+def test_ring_cut_is_invariant_under_rotation_of_the_embedding_and_keeps_groups_whole():
+    rng = np.random.default_rng(9)
+    ang = rng.uniform(-math.pi, math.pi, 60)
+    base = wo.cut_ring_at_largest_gap(wo.stage1_order(ang), ang)
+    wrap = lambda a: (a + math.pi) % (2 * math.pi) - math.pi
+    for theta in (0.3, 1.7, 3.0, -2.2):
+        rot = wrap(ang + theta)
+        assert wo.cut_ring_at_largest_gap(wo.stage1_order(rot), rot).tolist() == base.tolist()
+        # the plain -pi cut is not invariant: it starts wherever -pi happens to fall
+    assert any(wo.stage1_order(wrap(ang + t)).tolist() != wo.stage1_order(ang).tolist() for t in (0.3, 1.7))
+    # three tight groups, one of them straddling +-pi: the -pi cut splits it, the largest-gap cut does not
+    lab = np.repeat([0, 1, 2], 8)
+    centre = np.array([math.pi, -1.0, 1.0])
+    a = wrap(centre[lab] + rng.uniform(-0.05, 0.05, 24))
+    runs = lambda o: int((lab[o][1:] != lab[o][:-1]).sum())
+    assert runs(wo.stage1_order(a)) == 3
+    oc = wo.cut_ring_at_largest_gap(wo.stage1_order(a), a)
+    assert runs(oc) == 2
+    # with one wave per group the overlap score of identical-row groups can only gain
+    mk = np.zeros((24, 30), dtype=bool)
+    for g in range(3):
+        mk[lab == g, g * 10:(g + 1) * 10] = True
+    s_cut, s_pi = wo.scores(mk, oc, 8), wo.scores(mk, wo.stage1_order(a), 8)
+    assert s_cut["Ov"] > s_pi["Ov"] and s_cut["U"] < s_pi["U"]
+
+
+def test_plan_head_with_ring_cut_is_valid_and_not_worse_on_planted_masks():
+    mk, label = _planted(4, 12, 6, 3)
+    W = 12
+    a = wo.plan_head(mk, W, 40, 5, 0, mode=wo.MODE_FORCE_REORDER)
+    b = wo.plan_head(mk, W, 40, 5, 0, mode=wo.MODE_FORCE_REORDER, ring_cut=True)
+    assert sorted(b["row_order"].tolist()) == list(range(48))
+    assert np.array_equal(b["order1"], wo.cut_ring_at_largest_gap(a["order1"], a["angles"]))
+    assert np.array_equal(b["row_order"], wo.stage2_order(b["order1"], wo.row_nnz(mk), W))
+    sa, sb = wo.scores(mk, a["row_order"], W), wo.scores(mk, b["row_order"], W)
+    assert sb["Ov"] >= sa["Ov"] and sb["U"] <= sa["U"]
+    lab = label[b["order1"]]
+    assert int((lab[1:] != lab[:-1]).sum()) == 3            # every group in one piece
