@@ -184,9 +184,11 @@ def run_waveal(args, cfg):
     bitmap = bitmap_h.to(dev, non_blocking=True)
     ptr = torch.from_numpy(ptr_np).to(dev)
     idx = torch.from_numpy(idx_np).to(dev)
-    W = wb.default_wave_size()
+    W = args.wave if args.wave > 0 else wb.default_wave_size()
     step_mode = {"reorder": wb.FORCE_REORDER, "natural": wb.FORCE_NATURAL, "auto": wb.AUTO,
                  "stage1": wb.STAGE1_ONLY, "stage2": wb.STAGE2_ONLY}[args.plan_mode]
+    ring = wb.RING_CUT_LARGEST_GAP if args.ring_cut else 0
+    step_mode |= ring
     pdesc = wb.plan_desc_default(heads=H, n_q_blocks=nb, n_kv_blocks=nb, wave_size=W, mode=step_mode,
                                  seed=cfg.plan_seed, kv_bytes_per_head=2 * Sp * D * 2)
     if args.svd_iters > 0:
@@ -261,7 +263,7 @@ def run_waveal(args, cfg):
 
     # planned vs natural row order of the same kernel: interleaved launches, per-pair ratios,
     # and the kernel's own cycle counts (clock-independent)
-    pdesc.mode = wb.FORCE_REORDER
+    pdesc.mode = wb.FORCE_REORDER | ring
     reo = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream).row_order
     if sampler:
         torch.cuda.synchronize()
@@ -273,7 +275,7 @@ def run_waveal(args, cfg):
     check_status()
     t_reo, t_nat = ab["a_ms"], ab["b_ms"]
     t_plan = timed(lambda: wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream))
-    pdesc.mode = wb.AUTO
+    pdesc.mode = wb.AUTO | ring
     auto = wb.plan_bitmap(pdesc, bitmap, workspace=pws, stream=stream)
     torch.cuda.synchronize()
     skipped = int((auto.skip_flags & 1).sum().item())
@@ -383,7 +385,7 @@ def run_waveal(args, cfg):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "heads": cfg.heads, "heads_per_rank": H, "head_dim": D, "seq": S, "block": B,
                    "block_pairs_rank0": pairs,
-                   "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode, "heads_in_natural_order": step_skipped,
+                   "density": pairs / (H * nb * nb), "wave_size": W, "plan_mode": args.plan_mode, "ring_cut": bool(args.ring_cut), "heads_in_natural_order": step_skipped,
                    "mask": args.mask, "head_order": args.head_order, "svd_iters": int(pdesc.svd_iters),
                    "step": "plan + attention", "l2": "inputs (Q,K,V,O %.1f GB per rank) larger than L2, no flush" %
                    (4 * H * Sp * D * 2 / 1e9),
@@ -439,6 +441,8 @@ def main():
     ap.add_argument("--head-order", default="sequential", choices=["sequential", "interleaved"],
                     help="ticket order: all rows of a head before the next head, or position-major over heads")
     ap.add_argument("--svd-iters", type=int, default=0, help="T of Algorithm 1 (0 = the library default)")
+    ap.add_argument("--wave", type=int, default=0, help="W the plan buckets by (0 = the kernel's tasks in flight, SM count)")
+    ap.add_argument("--ring-cut", action="store_true", help="Stage-1 variant: open the angular ring at its largest gap")
     ap.add_argument("--ab-pairs", type=int, default=12, help="interleaved launch pairs of the planned-vs-natural comparison")
     ap.add_argument("--replicas", action="store_true", help="N > 1: every rank runs a whole batch element (weak scaling) "
                                                              "instead of a slice of the heads")

@@ -64,6 +64,13 @@ typedef enum {
   WAVEAL_STAGE2_ONLY = 4     /* natural order cut into waves, each sorted by block count   */
 } waveal_mode;
 
+/* Optional bit, OR-ed into waveal_plan_desc.mode: open the ring of angularly sorted rows at the
+ * largest gap between neighbouring angles instead of at -pi, where Eq. 4's atan2 puts the cut
+ * (Section 4.3.1 calls the sorted rows a ring but does not say where it is opened).  A variant
+ * for experiments, off by default: it makes Stage 1 invariant under rotations of the embedding
+ * and keeps a tight group of rows that straddles +-pi in one piece. */
+#define WAVEAL_RING_CUT_LARGEST_GAP 16
+
 /* skip_flags bits */
 #define WAVEAL_FLAG_SKIPPED 1u        /* this head's row_order is the identity (skip applied) */
 #define WAVEAL_FLAG_SHORT_SEQ 2u      /* one head's K+V fit the L2 budget (Section 4.5, case 1) */
@@ -76,7 +83,7 @@ typedef struct waveal_plan_desc {
   int32_t n_kv_blocks;    /* N_B                                                              */
   int32_t wave_size;      /* W = SMs x resident CTAs (Section 6.1); 0 = this device's SM count */
   int32_t svd_iters;      /* T of Algorithm 1 (paper: 5-15; library default 5)                */
-  int32_t mode;           /* waveal_mode                                                      */
+  int32_t mode;           /* waveal_mode, optionally | WAVEAL_RING_CUT_LARGEST_GAP            */
   uint64_t seed;          /* seed of the start block of Algorithm 1                           */
   /* guard thresholds, all integer comparisons (the "offline profile" of Section 4.5):       */
   int64_t kv_bytes_per_head; /* bytes of K plus V of one head; 0 disables the short-seq test */
@@ -175,6 +182,13 @@ size_t waveal_noalloc_max_rows(void);
  * through the common exit (no trap, no fault, the context stays usable); O is then undefined.
  * The next call on the same workspace works as usual. */
 #define WAVEAL_ATTN_SELFTEST_LOST_TILE 256
+/* 64-row query blocks run in a 128-row tensor-core tile.  By default two query blocks that stand
+ * at positions 2i and 2i+1 of a head's execution order and have the very same list of KV blocks
+ * (rows that attend to everything, duplicated rows) share one tile, which halves their cost;
+ * the results are the same bits as without sharing (the two blocks never interact: a row of the
+ * tile only sees its own row of Q).  Stage 2 of the plan puts such rows side by side, because
+ * it sorts a wave by block count.  This flag switches the sharing off (comparison runs). */
+#define WAVEAL_ATTN_NO_ROW_PAIRING 2
 
 typedef struct waveal_attn_desc {
   int32_t heads;            /* batch*heads; K/V heads == Q heads                              */
@@ -190,7 +204,7 @@ typedef struct waveal_attn_desc {
 /* Bytes of device workspace waveal_bsattn_fwd needs: 32 bytes of counters (int32 words: ticket
  * counter, abort flag, number of tasks computed twice, ticket counter of the second launch,
  * length of the first and of the second launch in SM cycles = the largest lifetime of a thread
- * block, two spare), 8 bytes per (head, query block) for the list of tasks to compute again and
+ * block, number of query-block pairs that shared a tile, one spare), 8 bytes per (head, query block) for the list of tasks to compute again and
  * 32 bytes per (head, query block) for the table that maps a ticket to its task.  The counters
  * are live state of the call (tickets are drawn from them): calls that may overlap on the GPU
  * must not share a workspace.  Host-only. */

@@ -245,8 +245,10 @@ def scatter_rows(src, dst, row_order, block: int, stream=None):
     _move_rows("waveal_scatter_rows", src, dst, row_order, block, stream)
 
 
+RING_CUT_LARGEST_GAP = 16
 ATTN_ONLINE_MAX_ONLY = 1
 ATTN_SELFTEST_LOST_TILE = 256
+ATTN_NO_ROW_PAIRING = 2
 
 
 def attn_desc(q, k, v, o, seq_q: int, seq_kv: int, block: int, interleaved: bool = False, flags: int = 0) -> AttnDesc:

@@ -269,8 +269,12 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool b_mn_major)
 // ------------------------------------------------------------------ kernel
 
 // n: KV tiles of the task (a tile = 128 keys = 128/block consecutive entries of the row's list),
-// len: entries of the list, tail_valid: keys of the last tile that exist
-struct Task { int h, row, lo, n, tail_valid, len, pad1, pad2; };
+// len: entries of the list, tail_valid: keys of the last tile that exist.
+// row2 (64-row query blocks only): a second query block with the very same list, or -1; its rows
+// fill the other half of the 128-row MMA tile, so the pair costs what one block costs.  The
+// ticket of the second block of a pair carries n = kAbsorbed and is skipped by whoever draws it.
+struct Task { int h, row, lo, n, tail_valid, len, row2, pad2; };
+constexpr int kAbsorbed = -2;
 
 // tiles, list length and valid keys of the last tile from a list of `len` blocks of `block` keys
 // whose last entry is `last`
@@ -301,6 +305,7 @@ struct AttnParams {
   long long total_tasks;
   long long wait_limit;   // cycles a bounded wait may take (kTimeoutCycles; far shorter under the self-test flag)
   int drop_tile;          // self-test: the producer never loads the first K tile of ticket 0
+  int no_pairing;         // 64-row blocks: never put two blocks with identical lists into one tile
   float sl2;          // scale * log2(e)
 };
 
@@ -474,12 +479,14 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         const uint4* e = reinterpret_cast<const uint4*>(p.table + t);
         const uint4 a = e[0], b = e[1];
         tk.h = (int)a.x; tk.row = (int)a.y; tk.lo = (int)a.z; tk.n = (int)a.w; tk.tail_valid = (int)b.x; tk.len = (int)b.y;
+        tk.row2 = (int)b.z;
+        if (tk.n == kAbsorbed) continue;          // second block of a pair: computed with its partner
       } else {
         int h = p.ws[8 + 2 * t], row = p.ws[9 + 2 * t];
         if (h < 0 || h >= p.heads) h = 0;
         if (row < 0 || row >= p.m_b) row = 0;
         int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
-        tk.h = h; tk.row = row; tk.lo = lo;
+        tk.h = h; tk.row = row; tk.lo = lo; tk.row2 = -1;
         fill_tiles(tk, max(hi - lo, 0), BLOCK, hi > lo ? p.kv_idx[hi - 1] : 0, p.n_b, p.seq_kv);
       }
       const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
@@ -496,10 +503,17 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       ok = warp_wait(ctx, BAR(B_Q_EMPTY), (q_it & 1) ^ 1, 2);
       if (!ok) break;
       if (lane == 0) {
-        mbar_expect_tx(BAR(B_Q_FULL), G::SLABS * G::BQ * 128);
+        const bool two = G::KB == 2 && tk.row2 >= 0;
+        mbar_expect_tx(BAR(B_Q_FULL), (two ? 2 : 1) * G::SLABS * G::BQ * 128);
 #pragma unroll
         for (int s = 0; s < G::SLABS; ++s)
           tma_load_3d(sbase + G::OFF_Q + s * 128 * 128, &tmQ, s * 64, tk.row * G::BQ, tk.h, BAR(B_Q_FULL));
+        if (two) {
+          // the partner's 64 rows go to rows 64..127 of the tile
+#pragma unroll
+          for (int s = 0; s < G::SLABS; ++s)
+            tma_load_3d(sbase + G::OFF_Q + s * 128 * 128 + 64 * 128, &tmQ, s * 64, tk.row2 * G::BQ, tk.h, BAR(B_Q_FULL));
+        }
       }
       q_armed = true; q_armed_parity = q_it & 1;
       ++q_it;
@@ -744,8 +758,10 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const uint32_t rslot = task_it & 1;
       ++task_it;
       if (tk.n < 0) break;
-      const long long q_tok = (long long)tk.row * G::BQ + r;
-      const bool row_live = r < G::BQ && q_tok < p.seq_q;
+      // rows 64..127 of the tile belong to the partner block of a pair (64-row blocks only)
+      const bool second = G::KB == 2 && r >= G::BQ;
+      const long long q_tok = second ? (long long)tk.row2 * G::BQ + (r - G::BQ) : (long long)tk.row * G::BQ + r;
+      const bool row_live = (second ? tk.row2 >= 0 : r < G::BQ) && q_tok < p.seq_q;
       __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + part * G::CO;
       if (tk.n == 0) {
         if (row_live) {
@@ -919,9 +935,10 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (FAST && sw == 0 && lane == 0 && redo_flag[rslot]) {
         // every warp's blocks of this task lie before O_FULL; the slot is used again two tasks
         // later, after this warp's O_FREE arrival below
-        const int e = atomicAdd(&p.ws[2], 1);
+        const int e = atomicAdd(&p.ws[2], (G::KB == 2 && tk.row2 >= 0) ? 2 : 1);
         p.ws[8 + 2 * e] = tk.h;
         p.ws[9 + 2 * e] = tk.row;
+        if (G::KB == 2 && tk.row2 >= 0) { p.ws[10 + 2 * e] = tk.h; p.ws[11 + 2 * e] = tk.row2; }   // computed again one by one
         redo_flag[rslot] = 0;
       }
       exb[part * 128 + r] = make_float2(m_ref, l_run);
@@ -1003,13 +1020,31 @@ __global__ void k_task_table(AttnParams p, int block_k, Task* table) {
   const int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
   if (lo < 0 || hi < lo || (long long)hi > nnz) { report(32, lo < 0 ? lo : hi); bad = true; }
   Task tk{};
-  tk.h = h; tk.row = row; tk.lo = bad ? 0 : lo;
+  tk.h = h; tk.row = row; tk.lo = bad ? 0 : lo; tk.row2 = -1;
   int len = bad ? 0 : hi - lo, last = 0;
   if (len > 0) {
     last = p.kv_idx[hi - 1];
     if (last < 0 || last >= p.n_b) { report(33, last); len = 0; }
   }
   fill_tiles(tk, len, block_k, last, p.n_b, p.seq_kv);
+  // 64-row query blocks: positions 2i and 2i+1 of a head's order whose lists are identical
+  // (rows that attend to everything, duplicated rows) share one 128-row tile.  Both threads of
+  // a pair run the same comparison; the even position keeps the task, the odd one is absorbed.
+  if (block_k == 64 && len > 0 && !bad && !p.no_pairing) {
+    const int pos2 = pos ^ 1;
+    if (pos2 < p.m_b) {
+      const int other = p.row_order ? p.row_order[(size_t)h * p.m_b + pos2] : pos2;
+      if (other >= 0 && other < p.m_b && other != row) {
+        const int lo2 = p.row_ptr[(size_t)h * p.m_b + other], hi2 = p.row_ptr[(size_t)h * p.m_b + other + 1];
+        bool same = lo2 >= 0 && hi2 - lo2 == len && (long long)hi2 <= nnz;
+        for (int e = 0; same && e < len; ++e) same = p.kv_idx[lo + e] == p.kv_idx[lo2 + e];
+        if (same) {
+          if (pos & 1) tk.n = kAbsorbed;
+          else { tk.row2 = other; atomicAdd(&p.ws[6], 1); }     // word 6: pairs formed by this call
+        }
+      }
+    }
+  }
   table[t] = tk;
 }
 
@@ -1084,11 +1119,12 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   Task* table = reinterpret_cast<Task*>(reinterpret_cast<char*>(p.ws) + table_offset(p.total_tasks));
   p.table = table;
   p.redo_pass = 0;
-  k_task_table<<<(unsigned)((p.total_tasks + 255) / 256), 256, 0, st>>>(p, BLOCK, table);
-  WAVEAL_CUDA_OK(cudaGetLastError());
   p.wait_limit = kTimeoutCycles;
   p.drop_tile = 0;
   if (d->flags & WAVEAL_ATTN_SELFTEST_LOST_TILE) { p.wait_limit = kSelfTestCycles; p.drop_tile = 1; }
+  p.no_pairing = (d->flags & WAVEAL_ATTN_NO_ROW_PAIRING) ? 1 : 0;
+  k_task_table<<<(unsigned)((p.total_tasks + 255) / 256), 256, 0, st>>>(p, BLOCK, table);
+  WAVEAL_CUDA_OK(cudaGetLastError());
   if (d->flags & WAVEAL_ATTN_ONLINE_MAX_ONLY) {
     p.redo_pass = 0;
     k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);

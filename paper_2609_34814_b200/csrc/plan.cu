@@ -366,6 +366,7 @@ struct PlanParams {
   const u64* M;
   const u64* Mt;
   int m_b, n_b, wq, wk, wave, iters, mode, n_pow2, state_in_smem;
+  int ring_cut;         // open the angular ring at its largest gap instead of at -pi
   u64 seed;
   long long kv_bytes, l2_bytes, min_nnz;
   int fit_num, fit_den, min_ppm, loc_num, loc_den;
@@ -532,6 +533,40 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_head(PlanParams p) {
     }
     __syncthreads();
     bitonic_sort(keys, vals, p.n_pow2);     // Stage 1: rows by ascending angle, ties by row index
+    if (p.ring_cut && m_b >= 2) {
+      // Variant: the sorted rows form a ring (Section 4.3.1); open it at the largest gap between
+      // neighbouring angles (the gap around the back, first + 2 pi - last, included; the first
+      // of equal gaps wins) instead of at -pi, where atan2 happens to put the cut.
+      auto angle_at = [&](int i) {          // inverse of sortable()
+        const u64 k = keys[i];
+        return __longlong_as_double((long long)((k >> 63) ? (k & 0x7FFFFFFFFFFFFFFFull) : ~k));
+      };
+      double best = -1.0;
+      for (int i = tid; i < m_b; i += kPlanThreads) {
+        const double g = i + 1 < m_b ? angle_at(i + 1) - angle_at(i)
+                                     : (angle_at(0) + 2.0 * 3.14159265358979323846) - angle_at(m_b - 1);
+        best = fmax(best, g);
+      }
+      best = block_max(best, scratch);
+      int at = INT_MAX;
+      for (int i = tid; i < m_b; i += kPlanThreads) {
+        const double g = i + 1 < m_b ? angle_at(i + 1) - angle_at(i)
+                                     : (angle_at(0) + 2.0 * 3.14159265358979323846) - angle_at(m_b - 1);
+        if (g == best) at = min(at, i);
+      }
+      at = block_min_int(at, reinterpret_cast<int*>(scratch));
+      // rotate: the row behind the gap comes first (the key array is free until Stage 2 refills it)
+      int* tmp = reinterpret_cast<int*>(keys);
+      __syncthreads();
+      for (int i = tid; i < m_b; i += kPlanThreads) {
+        int src = i + at + 1;
+        if (src >= m_b) src -= m_b;
+        tmp[i] = vals[src];
+      }
+      __syncthreads();
+      for (int i = tid; i < m_b; i += kPlanThreads) vals[i] = tmp[i];
+      __syncthreads();
+    }
   } else {
     if (p.embedding)
       for (int i = tid; i < m_b; i += kPlanThreads) { p.embedding[((size_t)h * m_b + i) * 2] = 0.0; p.embedding[((size_t)h * m_b + i) * 2 + 1] = 0.0; }
@@ -576,7 +611,8 @@ waveal_status plan_layout(const waveal_plan_desc* d, PlanLayout* L) {
     return waveal::fail(WAVEAL_ERR_INVALID_ARG, "heads, n_q_blocks and n_kv_blocks must be positive");
   if (d->wave_size < 0 || d->svd_iters < 0 || d->svd_iters > 1000)
     return waveal::fail(WAVEAL_ERR_INVALID_ARG, "wave_size must be >= 0 and svd_iters in [0, 1000]");
-  if (d->mode < WAVEAL_AUTO || d->mode > WAVEAL_STAGE2_ONLY)
+  const int base_mode = d->mode & ~WAVEAL_RING_CUT_LARGEST_GAP;
+  if (base_mode < WAVEAL_AUTO || base_mode > WAVEAL_STAGE2_ONLY)
     return waveal::fail(WAVEAL_ERR_INVALID_ARG, "unknown mode %d", d->mode);
   if (d->l2_fit_den <= 0 || d->local_den <= 0 || d->l2_fit_num < 0 || d->local_num < 0 || d->min_density_ppm < 0)
     return waveal::fail(WAVEAL_ERR_INVALID_ARG, "guard thresholds must be non-negative with positive denominators");
@@ -636,7 +672,8 @@ waveal_status plan_common(const waveal_plan_desc* d, const u64* mask_bits, const
   PlanParams p{};
   p.M = M; p.Mt = Mt; p.m_b = (int)m; p.n_b = (int)n; p.wq = L.wq; p.wk = L.wk;
   p.wave = d->wave_size > 0 ? d->wave_size : sms;
-  p.iters = d->svd_iters; p.mode = d->mode; p.n_pow2 = L.n_pow2; p.state_in_smem = L.state_in_smem;
+  p.iters = d->svd_iters; p.mode = d->mode & ~WAVEAL_RING_CUT_LARGEST_GAP;
+  p.ring_cut = (d->mode & WAVEAL_RING_CUT_LARGEST_GAP) ? 1 : 0; p.n_pow2 = L.n_pow2; p.state_in_smem = L.state_in_smem;
   p.seed = d->seed;
   p.kv_bytes = d->kv_bytes_per_head; p.l2_bytes = d->l2_bytes > 0 ? d->l2_bytes : (long long)l2;
   p.min_nnz = d->min_nnz; p.fit_num = d->l2_fit_num; p.fit_den = d->l2_fit_den; p.min_ppm = d->min_density_ppm;

@@ -396,3 +396,53 @@ def test_malformed_lists_are_reported_not_followed():
     w.idx = keep_idx
     o, st = run_attention(w, out=torch.zeros_like(w.o))
     assert st == [0, 0, 0, 0] and torch.equal(o, good)
+
+
+def test_identical_rows_share_a_tile_with_identical_bits():
+    """64-row query blocks with the very same KV list at positions 2i, 2i+1 of the order run as one
+    128-row tile: same bits as unshared, same as any other order, and equal to the oracle."""
+    cfg = _small("ltxmixed", 4, 2, cut=10)          # 64x64 blocks, ragged tail, sink rows (full lists)
+    w = Workload(cfg)
+    nb = cfg.n_blocks
+    # make sure identical lists exist beyond the sink rows: copy a few rows' lists
+    masks = [m.copy() for m in w.masks]
+    for m in masks:
+        m[11] = m[10]
+        m[nb - 1] = m[nb - 2]
+        m[21, :] = False
+        m[21, [3, 7]] = True                         # one tile, two blocks
+        m[20] = m[21]
+        m[31, :] = False
+        m[31, [5]] = True                            # half a tile
+        m[30] = m[31]
+    w.masks = masks
+    ptr, idx = I.masks_to_csr(masks)
+    w.ptr, w.idx = torch.from_numpy(ptr).cuda(), torch.from_numpy(idx).cuda()
+    b = cfg.block
+
+    def run(order, flags=0):
+        o = torch.full_like(w.o, float("nan"))
+        lse = torch.full((cfg.heads, cfg.seq), float("nan"), dtype=torch.float32, device="cuda")
+        d = wb.attn_desc(w.q, w.k, w.v, o, cfg.seq, cfg.seq, b, flags=flags)
+        ws = torch.zeros((wb.bsattn_workspace_bytes(d),), dtype=torch.uint8, device="cuda")
+        st = torch.zeros(4, dtype=torch.int32, device="cuda")
+        wb.bsattn_fwd(d, w.q, w.k, w.v, o, w.ptr, w.idx, row_order=order, lse=lse, workspace=ws, dev_status=st)
+        torch.cuda.synchronize()
+        assert st.tolist() == [0, 0, 0, 0]
+        return o, lse, int(ws.view(torch.int32)[6].item())
+
+    # Stage 2 (descending count inside a wave) puts the full rows side by side
+    d = wb.plan_desc_default(heads=cfg.heads, n_q_blocks=nb, n_kv_blocks=nb, wave_size=16, mode=wb.STAGE2_ONLY, seed=1)
+    plan = wb.plan_bitmap(d, w.bitmap if False else torch.from_numpy(
+        np.stack([I.mask_to_bitmap(m) for m in masks]).view(np.int64)).cuda())
+    shared, lse_s, pairs = run(plan.row_order)
+    alone, lse_a, none = run(plan.row_order, flags=wb.ATTN_NO_ROW_PAIRING)
+    natural, lse_n, pairs_nat = run(None)
+    assert none == 0 and pairs >= 4 and pairs_nat >= 4          # (10,11), (20,21), (30,31), the last two rows
+    assert torch.equal(shared[:, :cfg.seq], alone[:, :cfg.seq]) and torch.equal(lse_s, lse_a)
+    assert torch.equal(shared[:, :cfg.seq], natural[:, :cfg.seq]) and torch.equal(lse_s, lse_n)
+    assert torch.isnan(shared[:, cfg.seq:].float()).all()        # rows beyond the sequence stay untouched
+    for li in range(cfg.heads):
+        ref, ref_lse = _oracle_head(w, li)
+        assert_parity(shared[li, :cfg.seq].float().cpu().numpy(), ref, "shared tiles")
+        assert np.abs(lse_s[li].cpu().numpy() - ref_lse).max() < 2e-3

@@ -22,13 +22,13 @@ def _bitmap_dev(masks):
     return torch.from_numpy(bm.view(np.int64)).cuda()
 
 
-def _check_plan(masks, heads, wave, iters, seed, mode, res, guard=None, ov_tol=0.02):
+def _check_plan(masks, heads, wave, iters, seed, mode, res, guard=None, ov_tol=0.02, ring_cut=False):
     """Integer outputs bit-exact; Stage 1 by equality or by overlap score; Stage 2 bit-exact
     given the GPU's own Stage-1 order."""
     exact = 0
     for li, h in enumerate(heads):
         mk = masks[li]
-        ref = wo.plan_head(mk, wave, iters, seed, li, mode=mode, guard=guard)
+        ref = wo.plan_head(mk, wave, iters, seed, li, mode=mode, guard=guard, ring_cut=ring_cut)
         assert np.array_equal(_np(res.row_nnz[li]), ref["row_nnz"])
         assert np.array_equal(_np(res.col_count[li]), ref["col_count"])
         st = wo.guard_stats(mk, wave)
@@ -87,6 +87,30 @@ def test_plan_parity(name, frames, heads, wave):
     assert res.dev_status.tolist() == [0, 0, 0, 0]
     exact = _check_plan(masks, hs, wave, d.svd_iters, cfg.plan_seed, wo.MODE_FORCE_REORDER, res)
     assert exact >= 1          # fp64 on both sides: the permutation itself normally coincides
+
+
+@pytest.mark.parametrize("mode", [wb.FORCE_REORDER, wb.STAGE1_ONLY])
+def test_ring_cut_variant_matches_the_oracle(mode):
+    """Stage-1 variant: ring opened at the largest angular gap.  Same checks as the plain plan, plus:
+    the GPU's order1 is a rotation of the order1 it produces without the flag."""
+    cfg = I.scaled_config(I.CONFIGS["long720p"], frames=12)
+    hs = [0, 1, 2, 3]
+    masks = [I.make_mask(cfg, h) for h in hs]
+    bm = _bitmap_dev(masks)
+    d = wb.plan_desc_default(heads=4, n_q_blocks=cfg.n_blocks, n_kv_blocks=cfg.n_blocks, wave_size=32, mode=mode,
+                             seed=7, svd_iters=6)
+    plain = wb.plan_bitmap(d, bm, debug=True)
+    d.mode = mode | wb.RING_CUT_LARGEST_GAP
+    res = wb.plan_bitmap(d, bm, debug=True)
+    torch.cuda.synchronize()
+    exact = _check_plan(masks, hs, 32, 6, 7, mode, res, ring_cut=True)
+    assert exact >= 1
+    m = cfg.n_blocks
+    for li in range(4):
+        a, b = _np(plain.order1[li]).tolist(), _np(res.order1[li]).tolist()
+        assert any((a + a)[i:i + m] == b for i in range(m))
+        ang = np.arctan2(_np(res.embedding[li])[:, 1], _np(res.embedding[li])[:, 0])
+        assert b == wo.cut_ring_at_largest_gap(np.array(a), ang).tolist()
 
 
 @pytest.mark.parametrize("mode", [wb.STAGE1_ONLY, wb.STAGE2_ONLY, wb.FORCE_NATURAL, wb.AUTO])
