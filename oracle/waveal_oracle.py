@@ -17,7 +17,10 @@ Pins (tests/test_oracle_*.py): dense mask == textbook softmax attention and torc
 token-level brute force; closed forms; C twin (oracle_attn.c); Eq. 2 distance preservation;
 Eq. 3 against a LAPACK SVD; implicit centred products against the explicit centred matrix;
 subspace against numpy SVD on planted masks; Eq. 1 by brute-force pairwise distances;
-Stage 2 against Python's sorted(); the Section 4.4 example's ordering relations.
+Stage 2 against Python's sorted(); the Section 4.4 example's ordering relations; the start
+block against splitmix64's published outputs; the sign rule on hand-made vectors; the
+single-stage plan modes against the stage functions; the ring-cut variant by hand, as a
+rotation of the Stage-1 order and by its invariance under rotation of the embedding.
 Parity unpinned: the Stage-1 permutation at the working iteration count T (the paper prints
 no worked permutation); the guard's numeric thresholds (the paper gives none).
 """

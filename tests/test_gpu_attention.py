@@ -446,3 +446,14 @@ def test_identical_rows_share_a_tile_with_identical_bits():
         ref, ref_lse = _oracle_head(w, li)
         assert_parity(shared[li, :cfg.seq].float().cpu().numpy(), ref, "shared tiles")
         assert np.abs(lse_s[li].cpu().numpy() - ref_lse).max() < 2e-3
+    # a key far above the rest in a late block: tasks that share a tile are handed to the second
+    # launch as two single blocks, and the result still equals the unshared one and the oracle
+    k = w.k[0].float()
+    k[9 * b + 2] *= 300.0
+    w.k[0].copy_(k.to(torch.bfloat16))
+    shared, lse_s, pairs = run(plan.row_order)
+    alone, lse_a, _ = run(plan.row_order, flags=wb.ATTN_NO_ROW_PAIRING)
+    assert pairs >= 4 and torch.equal(shared[:, :cfg.seq], alone[:, :cfg.seq])
+    K64 = I.bf16_to_f64(w.k[0].cpu())
+    ref, _ = wo.block_sparse_attention(w.head_f64("q", 0), K64, w.head_f64("v", 0), masks[0], b, b, cfg.seq, cfg.seq)
+    assert_parity(shared[0, :cfg.seq].float().cpu().numpy(), ref, "shared tiles, second launch", one_hot=True)
