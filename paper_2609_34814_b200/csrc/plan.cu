@@ -7,11 +7,18 @@
 //   inside each bucket.
 //
 // Layout of the work: the mask is kept as a bitmap M and its bit transpose Mt (both stay
-// resident in L2; a bitmap is smaller than index lists once density exceeds 1/32).  One
-// CTA of 1024 threads owns one head and runs every step for it, with the iteration blocks
-// X, Y, Z (fp64) in shared memory, so the whole plan is one launch after the transpose and
-// no step needs a grid-wide barrier.  All floating-point reductions use a fixed thread ->
-// element assignment and a fixed combination tree, so a plan is reproducible bit for bit.
+// resident in L2; a bitmap is smaller than index lists once density exceeds 1/32).  A
+// thread-block cluster of 1 to 4 CTAs of 1024 threads (as many as the device holds at once
+// for the given number of heads) owns one head and runs every step for it, with the iteration
+// blocks X, Y, Z (fp64) in shared memory, so the whole plan is one launch after the transpose
+// and no step needs a grid-wide barrier.  The CTAs of a cluster keep identical copies of the
+// state: the cheap steps (counts, guard, QR, rotation) are done by each of them in the same
+// order, the two mask sweeps of an iteration - where the time goes - are split by rows and
+// each result is written into every copy through distributed shared memory; the lead CTA does
+// the sorts and writes the outputs.  All floating-point reductions use a fixed thread ->
+// element assignment and a fixed combination tree, and a row is summed by the same lanes in the
+// same order whichever CTA takes it, so a plan is reproducible bit for bit and does not
+// depend on the cluster size.
 #include <cfloat>
 #include <climits>
 #include <cmath>
@@ -205,6 +212,23 @@ __device__ __forceinline__ int block_min_int(int v, int* scratch) {
   return s;
 }
 
+// ---- thread-block cluster helpers: the CTAs of a cluster split the rows of the two mask sweeps
+// of a head between them and write every result into each other's shared memory
+__device__ __forceinline__ unsigned cluster_rank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// store a double2 at the same shared-memory offset of CTA `rank` of this cluster
+__device__ __forceinline__ void store_peer(const double2* local_ptr, unsigned rank, double2 v) {
+  unsigned laddr = (unsigned)__cvta_generic_to_shared(local_ptr), raddr;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(rank));
+  asm volatile("st.shared::cluster.v2.f64 [%0], {%1, %2};" ::"r"(raddr), "d"(v.x), "d"(v.y) : "memory");
+}
+
 // number of set bits with index in [lo, hi) of a bit row
 __device__ __forceinline__ int popcount_range(const u64* __restrict__ words, int lo, int hi) {
   if (hi <= lo) return 0;
@@ -222,14 +246,19 @@ __device__ __forceinline__ int popcount_range(const u64* __restrict__ words, int
 // L lanes share one bit row (lane q of the group takes words q, q+L, ...), 32/L rows per warp
 // step; the partial sums meet in a fixed shuffle tree of width L.  Fewer lanes per row than a
 // whole warp keeps more rows in flight and wastes fewer of the scarce fp64 adds on the tree.
+// crank / csize: this CTA's rank in its cluster and the cluster's size; the CTAs take the warp
+// steps in turn, and when `peers` is set (state in shared memory) every result is also written
+// into the other CTAs' copy of dst.  A row is summed by the same lanes in the same order
+// whichever CTA takes it, so the result does not depend on the cluster size.
 template <int L>
 __device__ __forceinline__ void gather_rows_l(const u64* __restrict__ bits, int n_rows, int wpr,
                                               const double2* src, double2* dst,
-                                              const int* __restrict__ cnt, double2 corr) {
+                                              const int* __restrict__ cnt, double2 corr,
+                                              int crank, int csize, bool peers) {
   constexpr int RPW = 32 / L;                       // rows per warp step
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = lane / L, q = lane % L;
-  for (int r0 = warp * RPW; r0 < n_rows; r0 += kPlanWarps * RPW) {
+  for (int r0 = (warp + crank * kPlanWarps) * RPW; r0 < n_rows; r0 += csize * kPlanWarps * RPW) {
     const int r = r0 + grp;
     const bool live = r < n_rows;
     double ax = 0.0, ay = 0.0;
@@ -265,21 +294,26 @@ __device__ __forceinline__ void gather_rows_l(const u64* __restrict__ bits, int 
     }
     if (live && q == 0) {
       const double sc = cnt ? (double)cnt[r] : 1.0;
-      dst[r] = make_double2(ax - sc * corr.x, ay - sc * corr.y);
+      const double2 v = make_double2(ax - sc * corr.x, ay - sc * corr.y);
+      dst[r] = v;
+      if (peers)
+        for (int c = 0; c < csize; ++c)
+          if (c != crank) store_peer(dst + r, (unsigned)c, v);
     }
   }
 }
 
 __device__ __forceinline__ void gather_rows(const u64* __restrict__ bits, int n_rows, int wpr,
                                             const double2* src, double2* dst,
-                                            const int* __restrict__ cnt, double2 corr) {
+                                            const int* __restrict__ cnt, double2 corr,
+                                            int crank, int csize, bool peers) {
   // about three words per lane
-  if (wpr <= 3) gather_rows_l<1>(bits, n_rows, wpr, src, dst, cnt, corr);
-  else if (wpr <= 6) gather_rows_l<2>(bits, n_rows, wpr, src, dst, cnt, corr);
-  else if (wpr <= 12) gather_rows_l<4>(bits, n_rows, wpr, src, dst, cnt, corr);
-  else if (wpr <= 24) gather_rows_l<8>(bits, n_rows, wpr, src, dst, cnt, corr);
-  else if (wpr <= 48) gather_rows_l<16>(bits, n_rows, wpr, src, dst, cnt, corr);
-  else gather_rows_l<32>(bits, n_rows, wpr, src, dst, cnt, corr);
+  if (wpr <= 3) gather_rows_l<1>(bits, n_rows, wpr, src, dst, cnt, corr, crank, csize, peers);
+  else if (wpr <= 6) gather_rows_l<2>(bits, n_rows, wpr, src, dst, cnt, corr, crank, csize, peers);
+  else if (wpr <= 12) gather_rows_l<4>(bits, n_rows, wpr, src, dst, cnt, corr, crank, csize, peers);
+  else if (wpr <= 24) gather_rows_l<8>(bits, n_rows, wpr, src, dst, cnt, corr, crank, csize, peers);
+  else if (wpr <= 48) gather_rows_l<16>(bits, n_rows, wpr, src, dst, cnt, corr, crank, csize, peers);
+  else gather_rows_l<32>(bits, n_rows, wpr, src, dst, cnt, corr, crank, csize, peers);
 }
 
 // Q factor of the thin QR of an m x 2 block: Gram-Schmidt with one re-orthogonalisation
@@ -367,6 +401,7 @@ struct PlanParams {
   const u64* Mt;
   int m_b, n_b, wq, wk, wave, iters, mode, n_pow2, state_in_smem;
   int ring_cut;         // open the angular ring at its largest gap instead of at -pi
+  int csize;            // CTAs per head (thread-block cluster size)
   u64 seed;
   long long kv_bytes, l2_bytes, min_nnz;
   int fit_num, fit_den, min_ppm, loc_num, loc_den;
@@ -381,7 +416,13 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_head(PlanParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   double* scratch = reinterpret_cast<double*>(smem);                 // (32 + 1) * 4 doubles
   unsigned char* region = smem + 2048;
-  const int h = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // A head is planned by a cluster of p.csize CTAs.  Everything cheap (counts, guard, QR,
+  // rotations, sorts) is done by every CTA of the cluster on its own copy of the state, in the
+  // same order, so the copies stay identical bit for bit; only the two mask sweeps of an
+  // iteration, where the time goes, are split, and their results exchanged.
+  const int csize = p.csize, crank = csize > 1 ? (int)cluster_rank() : 0;
+  const int h = blockIdx.x / csize, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool lead = crank == 0;         // writes the outputs
   const int m_b = p.m_b, n_b = p.n_b;
   const u64* M = p.M + (size_t)h * m_b * p.wq;
   const u64* Mt = p.Mt + (size_t)h * n_b * p.wk;
@@ -397,14 +438,14 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_head(PlanParams p) {
     for (int w = lane; w < p.wq; w += 32) c += __popcll(M[(size_t)r * p.wq + w]);
 #pragma unroll
     for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-    if (lane == 0) { nnz[r] = c; if (p.row_nnz) p.row_nnz[(size_t)h * m_b + r] = c; my_nnz += c; }
+    if (lane == 0) { nnz[r] = c; if (p.row_nnz && lead) p.row_nnz[(size_t)h * m_b + r] = c; my_nnz += c; }
   }
   for (int j = warp; j < n_b; j += kPlanWarps) {
     int c = 0;
     for (int w = lane; w < p.wk; w += 32) c += __popcll(Mt[(size_t)j * p.wk + w]);
 #pragma unroll
     for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-    if (lane == 0) { cnt[j] = c; if (p.col_count) p.col_count[(size_t)h * n_b + j] = c; }
+    if (lane == 0) { cnt[j] = c; if (p.col_count && lead) p.col_count[(size_t)h * n_b + j] = c; }
   }
   // ---- guard statistics over natural-order waves (Section 4.5)
   const int n_waves = (m_b + p.wave - 1) / p.wave;
@@ -430,11 +471,12 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_head(PlanParams p) {
   if (pair2 > 0 && 2 * ov * p.loc_den >= (long long)p.loc_num * pair2) flags |= WAVEAL_FLAG_ALREADY_LOCAL;
   const bool skip = p.mode == WAVEAL_FORCE_NATURAL || (p.mode == WAVEAL_AUTO && flags != 0);
   if (skip) flags |= WAVEAL_FLAG_SKIPPED;
-  if (tid == 0) {
+  if (tid == 0 && lead) {
     if (p.flags) p.flags[h] = (unsigned char)flags;
     if (p.stats) { long long* s = p.stats + (size_t)h * 4; s[0] = nnz_total; s[1] = ov; s[2] = pair2; s[3] = 0; }
   }
   if (skip) {
+    if (lead)
     for (int i = tid; i < m_b; i += kPlanThreads) {
       order_out[i] = i;
       if (order1_out) order1_out[i] = i;
@@ -465,16 +507,19 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_head(PlanParams p) {
     // ---- T sweeps + one more for the Rayleigh-Ritz step
     for (int it = 0; it <= p.iters; ++it) {
       // Y = M^T X - c (1^T X)/m
-      gather_rows(Mt, n_b, p.wk, X, Y, cnt, make_double2(colsum.x * inv_m, colsum.y * inv_m));
-      __syncthreads();
+      gather_rows(Mt, n_b, p.wk, X, Y, cnt, make_double2(colsum.x * inv_m, colsum.y * inv_m), crank, csize, csize > 1);
+      if (csize > 1) cluster_sync_all(); else __syncthreads();
       double cy[2] = {0, 0};
       for (int j = tid; j < n_b; j += kPlanThreads) { double2 y = Y[j]; double c = (double)cnt[j]; cy[0] += c * y.x; cy[1] += c * y.y; }
       block_sum<2>(cy, scratch);
       // Z = M Y - 1 (c^T Y)/m
-      gather_rows(M, m_b, p.wq, Y, Z, nullptr, make_double2(cy[0] * inv_m, cy[1] * inv_m));
-      __syncthreads();
+      gather_rows(M, m_b, p.wq, Y, Z, nullptr, make_double2(cy[0] * inv_m, cy[1] * inv_m), crank, csize, csize > 1);
+      if (csize > 1) cluster_sync_all(); else __syncthreads();
       if (it < p.iters) colsum = thin_qr2(Z, X, m_b, scratch);
     }
+    // the rest (ordering, angles, sorts, outputs) is cheap: the lead CTA finishes alone.  No CTA
+    // touches another's shared memory after the last exchange above.
+    if (!lead) return;
     // ---- B = X^T Z, rotate onto the eigenvectors of its symmetric part, larger Ritz value first
     double b[4] = {0, 0, 0, 0};
     for (int i = tid; i < m_b; i += kPlanThreads) {
@@ -568,6 +613,7 @@ __global__ void __launch_bounds__(kPlanThreads, 1) k_plan_head(PlanParams p) {
       __syncthreads();
     }
   } else {
+    if (!lead) return;
     if (p.embedding)
       for (int i = tid; i < m_b; i += kPlanThreads) { p.embedding[((size_t)h * m_b + i) * 2] = 0.0; p.embedding[((size_t)h * m_b + i) * 2 + 1] = 0.0; }
     for (int i = tid; i < p.n_pow2; i += kPlanThreads) vals[i] = i < m_b ? i : INT_MAX;
@@ -683,7 +729,28 @@ waveal_status plan_common(const waveal_plan_desc* d, const u64* mask_bits, const
   p.ws_state = reinterpret_cast<double2*>(w + L.off_state);
   p.row_order = out->row_order; p.row_nnz = out->row_nnz; p.flags = out->skip_flags; p.col_count = out->col_count;
   p.order1 = out->order1; p.embedding = out->embedding; p.stats = reinterpret_cast<long long*>(out->stats);
-  k_plan_head<<<(unsigned)H, kPlanThreads, L.smem, st>>>(p);
+  // CTAs per head: as many as fit the device at once (clusters of 1 to 4 CTAs on neighbouring
+  // SMs), when the iteration blocks live in shared memory and some head may be planned at all
+  int csize = 1;
+  if (L.state_in_smem && p.mode != WAVEAL_FORCE_NATURAL && p.mode != WAVEAL_STAGE2_ONLY) {
+    csize = (int)(sms / (long long)H);
+    csize = csize < 1 ? 1 : csize > 4 ? 4 : csize;
+  }
+  p.csize = csize;
+  if (csize == 1) {
+    k_plan_head<<<(unsigned)H, kPlanThreads, L.smem, st>>>(p);
+  } else {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(H * csize));
+    cfg.blockDim = dim3(kPlanThreads);
+    cfg.dynamicSmemBytes = L.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    WAVEAL_CUDA_OK(cudaLaunchKernelEx(&cfg, k_plan_head, p));
+  }
   ++launches;
   WAVEAL_CUDA_OK(cudaGetLastError());
   waveal::launch_counter() = launches;
