@@ -49,7 +49,8 @@ def ncu_counters(workload: str):
         for line in open(p):
             k, _, v = line.partition(":")
             if k in ("l2_hit_pct_reordered", "l2_hit_pct_natural", "dram_read_bytes_reordered",
-                     "dram_write_bytes_reordered", "dram_read_bytes_natural", "dram_write_bytes_natural"):
+                     "dram_write_bytes_reordered", "dram_read_bytes_natural", "dram_write_bytes_natural",
+                     "kernel_time_ns_natural", "kernel_time_ns_reordered"):
                 try:
                     out[k] = float(v.split()[0])
                 except (ValueError, IndexError):
@@ -382,6 +383,12 @@ def run_waveal(args, cfg):
     key = "natural" if step_skipped == H else "reordered" if step_skipped == 0 else "mixed"
     if f"dram_read_bytes_{key}" in ctr and f"dram_write_bytes_{key}" in ctr:
         traffic = ctr[f"dram_read_bytes_{key}"] + ctr[f"dram_write_bytes_{key}"]
+    for o in ("natural", "reordered"):
+        # achieved HBM rate of the captured launch against the measured copy bandwidth
+        if all(f"{x}_{o}" in ctr for x in ("dram_read_bytes", "dram_write_bytes", "kernel_time_ns")):
+            gbs = (ctr[f"dram_read_bytes_{o}"] + ctr[f"dram_write_bytes_{o}"]) / ctr[f"kernel_time_ns_{o}"]
+            ctr[f"hbm_gbs_{o}"] = gbs
+            ctr[f"hbm_frac_of_peak_{o}"] = gbs / pk["hbm"]
     clocks = sampler.summary("timed steps")
     clocks_ab = sampler.summary("order comparison")
     line = {
@@ -399,6 +406,7 @@ def run_waveal(args, cfg):
         "roofline": {"bound": "tensor", "kernel": "k_bsattn_fwd", "achieved": achieved, "peak": pk["bf16"],
                      "unit": "TFLOP/s", "frac": achieved / pk["bf16"], "peak_source": pk["source"] + " (burst)",
                      "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
+                     "frac_of_datasheet_2250": achieved / 2250.0,
                      "kernel_ms": attn_ms, "traffic": traffic,
                      "traffic_source": "ncu, one launch of this workload (profiles/)" if traffic else None},
         "counters": {"source": "profiles/k_bsattn_fwd_%s.txt (ncu, one launch per order)" % cfg.name, **ctr} if ctr else None,
