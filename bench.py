@@ -151,6 +151,8 @@ def run_waveal(args, cfg):
     rank, world, local = wd.init("nccl")
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the library has no CPU fallback")
+    if os.environ.get("WAVEAL_BENCH_ONE_DEVICE"):
+        local = 0                                 # functional test: all ranks share cuda:0 (control plane over gloo)
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     wb.load()

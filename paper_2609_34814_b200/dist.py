@@ -18,7 +18,11 @@ def env_rank() -> Tuple[int, int, int]:
 
 
 def init(backend: str = "nccl") -> Tuple[int, int, int]:
+    """Rendezvous of the launcher's ranks.  WAVEAL_DIST_BACKEND=gloo overrides the backend: the
+    control plane (barrier, max / sum of a scalar) then runs over gloo, which lets several ranks
+    share one GPU in a functional test - their kernels never wait on one another."""
     rank, world, local = env_rank()
+    backend = os.environ.get("WAVEAL_DIST_BACKEND", backend)
     if world > 1 and not dist.is_initialized():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29500")
@@ -42,10 +46,14 @@ def barrier():
         dist.barrier()
 
 
+def _scalar_device(device):
+    return "cpu" if dist.get_backend() == "gloo" else device
+
+
 def max_over_ranks(value: float, device="cpu") -> float:
     if not dist.is_initialized():
         return float(value)
-    t = torch.tensor([value], dtype=torch.float64, device=device)
+    t = torch.tensor([value], dtype=torch.float64, device=_scalar_device(device))
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
 
@@ -53,7 +61,7 @@ def max_over_ranks(value: float, device="cpu") -> float:
 def sum_over_ranks(value: float, device="cpu") -> float:
     if not dist.is_initialized():
         return float(value)
-    t = torch.tensor([value], dtype=torch.float64, device=device)
+    t = torch.tensor([value], dtype=torch.float64, device=_scalar_device(device))
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return float(t.item())
 
