@@ -182,12 +182,13 @@ size_t waveal_noalloc_max_rows(void);
  * through the common exit (no trap, no fault, the context stays usable); O is then undefined.
  * The next call on the same workspace works as usual. */
 #define WAVEAL_ATTN_SELFTEST_LOST_TILE 256
-/* 64-row query blocks run in a 128-row tensor-core tile.  By default two query blocks that stand
- * at positions 2i and 2i+1 of a head's execution order and have the very same list of KV blocks
- * (rows that attend to everything, duplicated rows) share one tile, which halves their cost;
- * the results are the same bits as without sharing (the two blocks never interact: a row of the
- * tile only sees its own row of Q).  Stage 2 of the plan puts such rows side by side, because
- * it sorts a wave by block count.  This flag switches the sharing off (comparison runs). */
+/* 64-row query blocks run in a 128-row tensor-core tile.  By default two query blocks of a head
+ * with the very same list of KV blocks share one tile, which halves their cost: rows that select
+ * every KV block pair up wherever they stand in the execution order (1st with 2nd, 3rd with 4th
+ * such row; the pair runs at the position of its first row), other rows when they stand at
+ * positions 2i and 2i+1 (Stage 2 of the plan puts rows of equal count side by side).  The results
+ * are the same bits as without sharing (the two blocks never interact: a row of the tile only
+ * sees its own row of Q).  This flag switches the sharing off (comparison runs). */
 #define WAVEAL_ATTN_NO_ROW_PAIRING 2
 
 typedef struct waveal_attn_desc {

@@ -1027,21 +1027,43 @@ __global__ void k_task_table(AttnParams p, int block_k, Task* table) {
     if (last < 0 || last >= p.n_b) { report(33, last); len = 0; }
   }
   fill_tiles(tk, len, block_k, last, p.n_b, p.seq_kv);
-  // 64-row query blocks: positions 2i and 2i+1 of a head's order whose lists are identical
-  // (rows that attend to everything, duplicated rows) share one 128-row tile.  Both threads of
-  // a pair run the same comparison; the even position keeps the task, the odd one is absorbed.
+  // 64-row query blocks: two blocks with the very same list share one 128-row tile.  Candidates:
+  //  - rows that select every KV block (list length = N_B: rows that attend to everything), wherever
+  //    they stand: the 1st and 2nd, the 3rd and 4th, ... such row of the head's order form pairs,
+  //    run at the position of the first of the two;
+  //  - any other two rows at positions 2i and 2i+1 of the order (Stage 2 of the plan puts rows of
+  //    equal count side by side).
+  // A pair is formed only if the two lists are equal entry by entry; both threads of a pair run
+  // the same comparison, the first keeps the task, the second one's ticket is absorbed.
   if (block_k == 64 && len > 0 && !bad && !p.no_pairing) {
-    const int pos2 = pos ^ 1;
-    if (pos2 < p.m_b) {
-      const int other = p.row_order ? p.row_order[(size_t)h * p.m_b + pos2] : pos2;
-      if (other >= 0 && other < p.m_b && other != row) {
-        const int lo2 = p.row_ptr[(size_t)h * p.m_b + other], hi2 = p.row_ptr[(size_t)h * p.m_b + other + 1];
-        bool same = lo2 >= 0 && hi2 - lo2 == len && (long long)hi2 <= nnz;
-        for (int e = 0; same && e < len; ++e) same = p.kv_idx[lo + e] == p.kv_idx[lo2 + e];
-        if (same) {
-          if (pos & 1) tk.n = kAbsorbed;
-          else { tk.row2 = other; atomicAdd(&p.ws[6], 1); }     // word 6: pairs formed by this call
-        }
+    const size_t hb = (size_t)h * p.m_b;
+    auto row_at = [&](int ps) {
+      const int r = p.row_order ? p.row_order[hb + ps] : ps;
+      return (r < 0 || r >= p.m_b) ? -1 : r;
+    };
+    auto len_of = [&](int r) { return p.row_ptr[hb + r + 1] - p.row_ptr[hb + r]; };
+    int mate = -1;            // the other row of the candidate pair
+    bool first = true;        // this thread's row is the first of the two
+    if (len == p.n_b) {
+      int before = 0;
+      for (int ps = 0; ps < pos; ++ps) { const int r = row_at(ps); if (r >= 0 && len_of(r) == p.n_b) ++before; }
+      first = (before & 1) == 0;
+      if (first) {
+        for (int ps = pos + 1; ps < p.m_b && mate < 0; ++ps) { const int r = row_at(ps); if (r >= 0 && len_of(r) == p.n_b) mate = r; }
+      } else {
+        for (int ps = pos - 1; ps >= 0 && mate < 0; --ps) { const int r = row_at(ps); if (r >= 0 && len_of(r) == p.n_b) mate = r; }
+      }
+    } else if ((pos ^ 1) < p.m_b) {
+      const int r = row_at(pos ^ 1);
+      if (r >= 0 && len_of(r) == len) { mate = r; first = (pos & 1) == 0; }
+    }
+    if (mate >= 0 && mate != row) {
+      const int lo2 = p.row_ptr[hb + mate], hi2 = p.row_ptr[hb + mate + 1];
+      bool same = lo2 >= 0 && hi2 - lo2 == len && (long long)hi2 <= nnz;
+      for (int e = 0; same && e < len; ++e) same = p.kv_idx[lo + e] == p.kv_idx[lo2 + e];
+      if (same) {
+        if (first) { tk.row2 = mate; atomicAdd(&p.ws[6], 1); }     // word 6: pairs formed by this call
+        else tk.n = kAbsorbed;
       }
     }
   }

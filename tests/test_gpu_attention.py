@@ -439,6 +439,9 @@ def test_identical_rows_share_a_tile_with_identical_bits():
     alone, lse_a, none = run(plan.row_order, flags=wb.ATTN_NO_ROW_PAIRING)
     natural, lse_n, pairs_nat = run(None)
     assert none == 0 and pairs >= 4 and pairs_nat >= 4          # (10,11), (20,21), (30,31), the last two rows
+    # rows that select every block pair up wherever they stand, also in natural order
+    full_pairs = sum(int((m.sum(axis=1) == nb).sum()) // 2 for m in masks)
+    assert full_pairs >= 2 and pairs_nat >= full_pairs and pairs >= full_pairs
     assert torch.equal(shared[:, :cfg.seq], alone[:, :cfg.seq]) and torch.equal(lse_s, lse_a)
     assert torch.equal(shared[:, :cfg.seq], natural[:, :cfg.seq]) and torch.equal(lse_s, lse_n)
     assert torch.isnan(shared[:, cfg.seq:].float()).all()        # rows beyond the sequence stay untouched
