@@ -460,3 +460,42 @@ def test_identical_rows_share_a_tile_with_identical_bits():
     K64 = I.bf16_to_f64(w.k[0].cpu())
     ref, _ = wo.block_sparse_attention(w.head_f64("q", 0), K64, w.head_f64("v", 0), masks[0], b, b, cfg.seq, cfg.seq)
     assert_parity(shared[0, :cfg.seq].float().cpu().numpy(), ref, "shared tiles, second launch", one_hot=True)
+
+
+@pytest.mark.parametrize("block,d", [(128, 128), (64, 128), (64, 64)])
+def test_different_query_and_key_lengths_and_the_single_launch_variant(block, d):
+    """M_B != N_B (the paper's problem statement allows it), both lengths ragged; the default two-launch
+    call and the variant that takes the max of every tile must both match the oracle."""
+    seq_q, seq_kv = 5 * block - 9, 11 * block - 37
+    mq, nk = 5, 11
+    rng = np.random.default_rng(block + d)
+    H = 2
+    g = torch.Generator().manual_seed(block * 7 + d)
+    q = torch.randn((H, mq * block, d), generator=g).to(torch.bfloat16)
+    k = torch.randn((H, nk * block, d), generator=g).to(torch.bfloat16)
+    v = torch.randn((H, nk * block, d), generator=g).to(torch.bfloat16)
+    masks = []
+    for h in range(H):
+        m = rng.random((mq, nk)) < 0.4
+        m[:, nk - 1] |= rng.random(mq) < 0.7          # the ragged last KV block is in most lists
+        m[np.arange(mq), np.arange(mq)] = True
+        m[1] = True                                    # a row that selects everything
+        m[3] = True                                    # and a second one: they share a tile on 64-row blocks
+        masks.append(m)
+    ptr_np, idx_np = I.masks_to_csr(masks)
+    ptr, idx = torch.from_numpy(ptr_np).cuda(), torch.from_numpy(idx_np).cuda()
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    for flags in (0, wb.ATTN_ONLINE_MAX_ONLY):
+        o = torch.full_like(qd, float("nan"))
+        lse = torch.full((H, seq_q), float("nan"), dtype=torch.float32, device="cuda")
+        desc = wb.attn_desc(qd, kd, vd, o, seq_q, seq_kv, block, flags=flags)
+        st = torch.zeros(4, dtype=torch.int32, device="cuda")
+        wb.bsattn_fwd(desc, qd, kd, vd, o, ptr, idx, lse=lse, dev_status=st)
+        torch.cuda.synchronize()
+        assert st.tolist() == [0, 0, 0, 0]
+        for h in range(H):
+            Q64, K64, V64 = (I.bf16_to_f64(t[h]) for t in (q, k, v))
+            ref, ref_lse = wo.block_sparse_attention(Q64, K64, V64, masks[h], block, block, seq_q, seq_kv)
+            assert_parity(o[h, :seq_q].float().cpu().numpy(), ref, f"{block}x{d} flags {flags}")
+            assert np.abs(lse[h].cpu().numpy() - ref_lse).max() < 2e-3
+            assert torch.isnan(o[h, seq_q:].float()).all()
