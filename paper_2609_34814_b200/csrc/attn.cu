@@ -11,9 +11,8 @@
 // Structure of one CTA (608 threads):
 //   warp 0      producer: takes tickets, publishes tasks, issues TMA loads of the Q tile and
 //               of the K and V tiles (128-byte-swizzled slabs) into two shared-memory rings
-//   warp 18     MMA issuer 1: S_j = Q K_j^T (operands in shared memory) into one of the S buffers
-//               in tensor memory (three for 128-row query blocks, with P written over S; two
-//               plus two P buffers for 64-row query blocks: see Geo), ahead of the softmax
+//   warp 18     MMA issuer 1: S_j = Q K_j^T (operands in shared memory) into one of three S
+//               buffers in tensor memory, up to three blocks ahead of the softmax
 //   warp 1      MMA issuer 2: O += P_j V_j (P read from tensor memory, where it lies over the
 //               columns S_j came from), fp32 accumulator in tensor memory.  Two issuing warps:
 //               the waits and ring arithmetic of one run while the other's MMAs execute
@@ -326,18 +325,7 @@ struct Geo {
   static constexpr int NSTAGE = NSTAGE_RAW > 8 ? 8 : NSTAGE_RAW;
   static constexpr int NKS = (NSTAGE + 1) / 2;       // K tile ring
   static constexpr int NVS = NSTAGE / 2;             // V tile ring
-  // Two arrangements of tensor memory and of the hand-over of its buffers:
-  //  - 128-row query blocks: three S buffers; P of a tile is written over the first half of its own
-  //    S columns and the buffer goes back to Q K^T when the tile's P V has completed; the softmax
-  //    teams take the tiles of a task in turn;
-  //  - 64-row query blocks (SEP_P): two S buffers, one per softmax team, and two separate P
-  //    buffers; an S buffer goes back to Q K^T as soon as its team has loaded the scores, a P
-  //    buffer to the team when the P V that read it has completed.  Fewer tiles in flight, but a
-  //    team's next scores are computed while it still works on the current tile; measured 14 %
-  //    fewer cycles on the 64-row shape and 5 % more on the 128-row shape, hence the split.
-  static constexpr bool SEP_P = KB == 2;
-  static constexpr int NSBUF = SEP_P ? 2 : 3;        // S buffers in tensor memory
-  static constexpr int KAHEAD = 3;                   // K tiles requested ahead of the V tiles
+  static constexpr int NSBUF = 3;                    // S/P buffers in tensor memory
   static constexpr int HC = BK / 2;                  // S columns of a row one softmax thread owns (a row has two owners)
   static constexpr int CH = 32;                      // S columns a softmax thread holds at a time
   static constexpr int NCH = HC / CH;                // such chunks per thread and block
@@ -346,13 +334,13 @@ struct Geo {
   static constexpr int OFF_K = OFF_Q + Q_BYTES;
   static constexpr int OFF_V = OFF_K + NKS * TILE_BYTES;
   static constexpr int OFF_BAR = OFF_V + NVS * TILE_BYTES;
-  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 5 * NSBUF + 2 + 2 + 8 + 4 + 8;
+  static constexpr int N_BAR = 4 + 2 + 2 * NKS + 2 * NVS + 4 * NSBUF + 2 + 2 + 8 + 4 + 8;
   static constexpr int OFF_TASK = OFF_BAR + ((N_BAR * 8 + 15) / 16) * 16;
   static constexpr int OFF_MX = OFF_TASK + 2 * (int)sizeof(Task);
   static constexpr int OFF_MISC = OFF_MX + 4 * 128 * 4 + 2 * 2 * 2 * 128 * 4 + 2 * 4 * 128 * 8;
   static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;   // + slack for 1024-byte alignment
-  // tensor memory: the S buffers of 128 columns, (SEP_P: two P buffers of 64,) then the output accumulator
-  static constexpr uint32_t S_STRIDE = 128, P_COL = 256, P_STRIDE = 64, O_COL = 384, TMEM_COLS = 512;
+  // tensor memory: three S/P buffers of 128 columns, then the output accumulator
+  static constexpr uint32_t S_STRIDE = 128, O_COL = 384, TMEM_COLS = 512;
 };
 
 struct Ctx {
@@ -412,8 +400,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   constexpr int B_TASK_FULL = 0, B_TASK_EMPTY = 2, B_Q_FULL = 4, B_Q_EMPTY = 5, B_K_FULL = 6,
                 B_K_EMPTY = B_K_FULL + G::NKS, B_V_FULL = B_K_EMPTY + G::NKS, B_V_EMPTY = B_V_FULL + G::NVS,
                 B_S_FULL = B_V_EMPTY + G::NVS, B_P_FULL = B_S_FULL + G::NSBUF, B_S_FREE = B_P_FULL + 2 * G::NSBUF,
-                B_P_FREE = B_S_FREE + G::NSBUF,
-                B_O_FULL = B_P_FREE + G::NSBUF, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1, B_MX = B_FINAL + 2,
+                B_O_FULL = B_S_FREE + G::NSBUF, B_O_FREE = B_O_FULL + 1, B_FINAL = B_O_FREE + 1, B_MX = B_FINAL + 2,
                 B_EX = B_MX + 8, B_HX = B_EX + 4;
   static_assert(B_HX + 8 <= G::N_BAR, "barrier count");
   Task* tasks = reinterpret_cast<Task*>(smem + G::OFF_TASK);
@@ -437,8 +424,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       mbar_init(BAR(B_S_FULL + i), 1);
       mbar_init(BAR(B_P_FULL + 2 * i), 4);      // one per half of P (the four warps that own that half in the block's team)
       mbar_init(BAR(B_P_FULL + 2 * i + 1), 4);
-      mbar_init(BAR(B_S_FREE + i), G::SEP_P ? 8 : 1);   // SEP_P: the eight warps of the buffer's team have read S; else: P V completed
-      mbar_init(BAR(B_P_FREE + i), 1);                  // SEP_P: P V of the tile has completed
+      mbar_init(BAR(B_S_FREE + i), 1);
     }
     mbar_init(BAR(B_O_FULL), 1);
     mbar_init(BAR(B_O_FREE), 16);
@@ -583,10 +569,10 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         else { v_armed |= 1u << st; v_parity = (v_parity & ~(1u << st)) | (sph << st); ++v_it; }
         return true;
       };
-      for (int j = 0; j < G::KAHEAD && j < tk.n && ok; ++j) ok = load_tile(true, j);
+      for (int j = 0; j < G::NSBUF && j < tk.n && ok; ++j) ok = load_tile(true, j);
       for (int j = 0; j < tk.n && ok; ++j) {
         ok = load_tile(false, j);
-        if (ok && j + G::KAHEAD < tk.n) ok = load_tile(true, j + G::KAHEAD);
+        if (ok && j + G::NSBUF < tk.n) ok = load_tile(true, j + G::NSBUF);
       }
     }
     if (*abort_smem) {
@@ -635,9 +621,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       for (int j = 0; j < n && ok; ++j) {
         ok = warp_wait(ctx, BAR(B_K_FULL + k_st), k_ph, 12);
         if (!ok) break;
-        // S[sb] is free again when the tile that used it last has let go of it: its P V completed
-        // (P lies in the buffer), or - SEP_P - its softmax team has loaded the scores (that event
-        // is phase number uses-1 of the buffer's barrier)
+        // S[sb] also holds the P tile of the block that used it last: wait until that block's
+        // P V has completed (its commit is phase number uses-1 of the buffer's barrier)
         if (first_uses > 0) {
           --first_uses;
         } else {
@@ -697,7 +682,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         // with its own barrier: the MMAs on the first half run while the softmax team is still
         // computing the second
         const uint64_t vd = vdesc0 + (uint64_t)(v_st * (uint32_t)(G::TILE_BYTES >> 4));
-        const uint32_t pbase = G::SEP_P ? tmem_base + G::P_COL + sb * G::P_STRIDE : tmem_base + sb * G::S_STRIDE;
+        const uint32_t pbase = tmem_base + sb * G::S_STRIDE;
         const uint32_t d_o = tmem_base + G::O_COL;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -718,14 +703,13 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           for (int kk = 0; kk < G::BK / 32; ++kk) {
             const int k = h * (G::BK / 32) + kk;
             // P of key half h lies over the first columns of that half's own S columns
-            // (SEP_P: in columns 32h .. 32h+31 of the tile's P buffer)
-            umma_bf16_ts(d_o, pbase + h * (G::SEP_P ? G::HC / 2 : G::HC) + kk * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+            umma_bf16_ts(d_o, pbase + h * G::HC + kk * 8, vd + (uint64_t)((k * 16 * 128) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
           }
         }
         if (!ok) break;
         {
           tc_commit(BAR(B_V_EMPTY + v_st));
-          tc_commit(BAR((G::SEP_P ? B_P_FREE : B_S_FREE) + sb));
+          tc_commit(BAR(B_S_FREE + sb));
           if (j == n - 1) tc_commit(BAR(B_O_FULL));
         }
         if (++v_st == (uint32_t)G::NVS) { v_st = 0; v_ph ^= 1; }
@@ -761,7 +745,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const uint32_t o_row = tmem_base + lane_addr + G::O_COL;
     const int part = team * 2 + half;
-    uint32_t task_it = 0, s_phase = 0, o_it = 0, mx_phase = 0, hx_it = 0, sb = 0, g = 0;   // s_phase bit b: parity of the uses of S[b] so far; g: tiles so far
+    uint32_t task_it = 0, s_phase = 0, o_it = 0, mx_phase = 0, hx_it = 0, sb = 0;   // s_phase bit b: parity of the uses of S[b] so far
     bool ok = true;
     while (ok) {
       const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
@@ -790,15 +774,12 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       // l_run: sum over this thread's columns of this team's blocks, relative to the reference m_ref
       float m_ref = -INFINITY, l_run = 0.f;
       for (int j = 0; j < tk.n && ok; ++j) {
-        // which team takes the tile: in turn inside a task, or - SEP_P - the team that owns the
-        // tile's S buffer (buffers and teams then alternate over the CTA's whole life)
-        const uint32_t par = G::SEP_P ? sb : ((uint32_t)j & 1u);
+        const uint32_t par = (uint32_t)j & 1u;
         if ((int)par == team) {
           ok = warp_wait(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
           if (!ok) break;
           tc_fence_after();
           const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE + half * G::HC;
-          const uint32_t p_addr = G::SEP_P ? tmem_base + lane_addr + G::P_COL + sb * G::P_STRIDE + half * (G::HC / 2) : s_addr;
           const bool ragged = j == tk.n - 1 && tk.tail_valid < G::BK;
           const int col0 = half * G::HC;       // first key of the block this thread looks at
           // ---- pass 1: row max (the values are loaded again for the exponentials: a second
@@ -877,7 +858,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           // the row's output columns.
           if (grow && j > 0) {
             const uint32_t sbp = sb == 0 ? (uint32_t)G::NSBUF - 1u : sb - 1u;
-            ok = warp_wait(ctx, BAR((G::SEP_P ? B_P_FREE : B_S_FREE) + sbp), ((s_phase >> sbp) & 1u) ^ 1u, 22);
+            ok = warp_wait(ctx, BAR(B_S_FREE + sbp), ((s_phase >> sbp) & 1u) ^ 1u, 22);
             if (!ok) break;
             tc_fence_after();
             const float alpha = ex2(m_prev - m_new);
@@ -906,12 +887,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             uint32_t sv[G::CH];
             WAVEAL_TMEM_LD32(s_addr + ch * G::CH, sv, 0);
             WAVEAL_TMEM_WAIT_LD32(sv, 0);
-            if (G::SEP_P && ch == G::NCH - 1) {
-              // the last read of S: the buffer may take the team's next tile
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(BAR(B_S_FREE + sb));
-            }
             if (ragged) {
 #pragma unroll
               for (int c = 0; c < G::CH; ++c)
@@ -931,15 +906,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
               fadd2(ls4[c & 2], ls4[(c & 2) + 1], ls4[c & 2], ls4[(c & 2) + 1], e0, e1);
               pk[c / 2] = __byte_perm(__float_as_uint(e0), __float_as_uint(e1), 0x7632);
             }
-            if (G::SEP_P && ch == 0 && g >= (uint32_t)G::NSBUF) {
-              // the P V of the team's previous tile (issued when this tile began) has left the buffer
-              ok = warp_wait(ctx, BAR(B_P_FREE + sb), ((s_phase >> sb) & 1u) ^ 1u, 27);
-              if (!ok) break;
-              tc_fence_after();
-            }
-            WAVEAL_TMEM_ST16(p_addr + ch * 16, pk, 0);
+            WAVEAL_TMEM_ST16(s_addr + ch * 16, pk, 0);
           }
-          if (!ok) break;
           const float l_blk = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
           l_run += l_blk;
           // all terms are positive (the transcendental unit returns +inf on overflow, the
@@ -953,7 +921,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb * 2 + half));
         }
         // both teams count every block
-        ++g;
         s_phase ^= 1u << sb;
         if (!(FAST && j >= 2)) mx_phase ^= 1u << par;   // one flip per arrival on that parity's barrier
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
