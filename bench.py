@@ -225,7 +225,6 @@ def run_waveal(args, cfg):
     # ---- timed region: K steps, events on the launching stream; the attention kernel of each
     #      step is bracketed by its own events for the roofline figure
     attn_ev = []
-    cyc_log = torch.zeros((args.steps,), dtype=torch.int32, device=dev)
     wd.barrier()
     torch.cuda.synchronize()
     sampler = wt.ClockSampler(local) if rank == 0 else None
@@ -250,6 +249,8 @@ def run_waveal(args, cfg):
     total_ms = wd.max_over_ranks(e0.elapsed_time(e1), dev)
     ms_per_step = total_ms / args.steps
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_ev)
+    step_cycles = int(aws_words[4].item())          # SM cycles of the attention launch of the last timed step
+    step_pairs = int(aws_words[6].item())           # query-block pairs that shared a tile in it (64-row blocks)
     check_status()
     flops_all = wd.sum_over_ranks(flops, dev) if world > 1 else flops
     value = flops_all / (ms_per_step * 1e-3) / 1e12
@@ -409,7 +410,8 @@ def run_waveal(args, cfg):
                      "unit": "TFLOP/s", "frac": achieved / pk["bf16"], "peak_source": pk["source"] + " (burst)",
                      "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
                      "frac_of_datasheet_2250": achieved / 2250.0,
-                     "kernel_ms": attn_ms, "traffic": traffic,
+                     "kernel_ms": attn_ms, "kernel_sm_cycles": step_cycles, "tiles_shared_by_two_blocks": step_pairs,
+                     "traffic": traffic,
                      "traffic_source": "ncu, one launch of this workload (profiles/)" if traffic else None},
         "counters": {"source": "profiles/k_bsattn_fwd_%s.txt (ncu, one launch per order)" % cfg.name, **ctr} if ctr else None,
         "kernel": {"attn_ms_reordered": t_reo, "attn_ms_natural": t_nat,
