@@ -481,6 +481,8 @@ def test_different_query_and_key_lengths_and_the_single_launch_variant(block, d)
         m[np.arange(mq), np.arange(mq)] = True
         m[1] = True                                    # a row that selects everything
         m[3] = True                                    # and a second one: they share a tile on 64-row blocks
+        if h == 1:
+            m[:] = True                                # all five rows full: two pairs and one block on its own
         masks.append(m)
     ptr_np, idx_np = I.masks_to_csr(masks)
     ptr, idx = torch.from_numpy(ptr_np).cuda(), torch.from_numpy(idx_np).cuda()
