@@ -177,8 +177,8 @@ size_t waveal_noalloc_max_rows(void);
  * the first K tile of the first task and every bounded wait gives up after about 2 ms instead
  * of 2 s.  The call must come back with dev_status = {WAVEAL_ERR_TIMEOUT, site, ...} - the
  * site is the first of the waits behind that tile to run out: 12 (the Q K^T issuer waiting for
- * the tile), 3 (the loader waiting for its ring slot), 14 or 21 (the P V issuer and the softmax
- * warps waiting for what the product would have fed them) - with all thread blocks leaving
+ * the tile), 3 or 4 (the K or the V loader waiting for a ring slot), 14 or 21 (the P V issuer and
+ * the softmax warps waiting for what the product would have fed them) - with all thread blocks leaving
  * through the common exit (no trap, no fault, the context stays usable); O is then undefined.
  * The next call on the same workspace works as usual. */
 #define WAVEAL_ATTN_SELFTEST_LOST_TILE 256

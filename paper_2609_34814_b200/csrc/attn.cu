@@ -39,8 +39,9 @@
 
 namespace {
 
-constexpr int kThreads = 608;
-constexpr int kProducerWarp = 0, kPvWarp = 1, kSoftmaxWarp0 = 2, kQkWarp = 18;
+// 19 warps, and a 20th (the V tile loader) in the kernels of the 64-row blocks
+template <int BLOCK> constexpr int kThreadsOf = BLOCK == 64 ? 640 : 608;
+constexpr int kProducerWarp = 0, kPvWarp = 1, kSoftmaxWarp0 = 2, kQkWarp = 18, kVLoadWarp = 19;
 constexpr long long kTimeoutCycles = 4000000000ll;   // ~2 s at boost clock
 constexpr long long kSelfTestCycles = 4000000ll;     // ~2 ms: wait limit under WAVEAL_ATTN_SELFTEST_LOST_TILE
 #ifndef WAVEAL_POLY_EVERY
@@ -326,6 +327,7 @@ struct Geo {
   static constexpr int NKS = (NSTAGE + 1) / 2;       // K tile ring
   static constexpr int NVS = NSTAGE / 2;             // V tile ring
   static constexpr int NSBUF = 3;                    // S/P buffers in tensor memory
+  static constexpr bool SPLIT_LOADERS = KB == 2;     // K and V tiles requested by a warp each (else one warp, interleaved)
   static constexpr int HC = BK / 2;                  // S columns of a row one softmax thread owns (a row has two owners)
   static constexpr int CH = 32;                      // S columns a softmax thread holds at a time
   static constexpr int NCH = HC / CH;                // such chunks per thread and block
@@ -381,10 +383,68 @@ __device__ __forceinline__ bool warp_wait(const Ctx& c, uint32_t bar, uint32_t p
   return __all_sync(0xffffffffu, mbar_wait(c, bar, parity, site));
 }
 
+// One K or V tile of a task into its ring stage (called by a whole warp).  Tile j covers entries
+// KB*j .. of the row's list (the last tile of an odd list of 64-key blocks has one block).
+// State of the caller: it (tiles loaded so far), armed / parity (per stage: a load is in flight,
+// and the parity its barrier completes with), chunk_base / my_idx (32 list entries at a time,
+// one per lane).  dropped: self-test of the abort path, the tile is never requested.
+template <class G, int BLOCK, bool IS_K>
+__device__ __forceinline__ bool load_kv_tile(const Ctx& ctx, const AttnParams& p, const Task& tk, bool dropped, int j,
+                                             int lane, uint32_t sbase, uint32_t bar_full0, uint32_t bar_empty0,
+                                             const CUtensorMap* tm, const CUtensorMap* tm2, uint32_t& it,
+                                             uint32_t& armed, uint32_t& parity, int& chunk_base, int& my_idx) {
+  constexpr uint32_t NST = IS_K ? G::NKS : G::NVS;
+  auto entry = [&](int q) -> int {
+    if (q < chunk_base || q >= chunk_base + 32) {
+      chunk_base = q & ~31;
+      const int e = chunk_base + lane;
+      my_idx = e < tk.len ? p.kv_idx[tk.lo + e] : 0;
+    }
+    int blk = __shfl_sync(0xffffffffu, my_idx, q - chunk_base);
+    if (blk < 0 || blk >= p.n_b) {                   // malformed list: report it and stay in range
+      if (lane == 0 && p.dev_status && atomicCAS(p.dev_status, 0, WAVEAL_ERR_BAD_MASK) == 0) {
+        p.dev_status[1] = 30; p.dev_status[2] = tk.h; p.dev_status[3] = blk;
+      }
+      blk = 0;
+    }
+    return blk;
+  };
+  const int nblk = G::KB == 1 ? 1 : min(G::KB, tk.len - G::KB * j);
+  int blk[G::KB];
+#pragma unroll
+  for (int e = 0; e < G::KB; ++e) blk[e] = e < nblk ? entry(G::KB * j + e) : 0;
+  const uint32_t st = it % NST, sph = (it / NST) & 1;
+  const uint32_t b_full = bar_full0 + 8u * st, b_empty = bar_empty0 + 8u * st;
+  if (!warp_wait(ctx, b_empty, sph ^ 1, IS_K ? 3 : 4)) return false;
+  ++it;
+  if (dropped) return true;
+  // one lane per box: lane e*SLABS + s requests slab s of block e
+  if (lane == 0) mbar_expect_tx(b_full, (uint32_t)nblk * G::SLABS * BLOCK * 128);
+  __syncwarp();
+  const uint32_t dst = sbase + (IS_K ? G::OFF_K : G::OFF_V) + st * G::TILE_BYTES;
+  const int e = lane / G::SLABS, sl = lane % G::SLABS;
+  // two 64-key blocks that follow each other in memory come as one box of 128 rows per slab
+  const bool joined = G::KB == 2 && nblk == 2 && blk[G::KB - 1] == blk[0] + 1;
+  if (joined) {
+    if (e == 0) tma_load_3d(dst + sl * G::KV_SLAB_BYTES, tm2, sl * 64, blk[0] * BLOCK, tk.h, b_full);
+  } else {
+    int my_blk = blk[0];
+#pragma unroll
+    for (int i = 1; i < G::KB; ++i) if (e == i) my_blk = blk[i];
+    if (e < nblk) tma_load_3d(dst + sl * G::KV_SLAB_BYTES + e * BLOCK * 128, tm, sl * 64, my_blk * BLOCK, tk.h, b_full);
+  }
+  armed |= 1u << st;
+  parity = (parity & ~(1u << st)) | (sph << st);
+  return true;
+}
+
 template <int BLOCK, int D, bool FAST>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsOf<BLOCK>, 1)
 k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-             const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+             const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmK2,
+             const __grid_constant__ CUtensorMap tmV2, const AttnParams p) {
+  // tmK2 / tmV2: the same K and V with boxes of 128 rows, used by the 64-key-block kernels when the
+  // two blocks of a tile lie next to each other in memory (for 128-key blocks they equal tmK / tmV)
   using G = Geo<BLOCK, D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -414,8 +474,8 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const long long t_start = clock64();
 
   if (tid == 0) {
-    // a task is read by the two MMA issuers and the sixteen softmax warps
-    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_TASK_FULL + i), 1); mbar_init(BAR(B_TASK_EMPTY + i), 18); }
+    // a task is read by the V loader, the two MMA issuers and the sixteen softmax warps
+    for (int i = 0; i < 2; ++i) { mbar_init(BAR(B_TASK_FULL + i), 1); mbar_init(BAR(B_TASK_EMPTY + i), G::SPLIT_LOADERS ? 19 : 18); }
     mbar_init(BAR(B_Q_FULL), 1);
     mbar_init(BAR(B_Q_EMPTY), 1);
     for (int i = 0; i < G::NKS; ++i) { mbar_init(BAR(B_K_FULL + i), 1); mbar_init(BAR(B_K_EMPTY + i), 1); }
@@ -440,7 +500,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     fence_proxy_async();
   }
   // the MMA reads all 128 rows of the Q region even when a query block has 64 rows: clear it once
-  for (int i = tid; i < G::Q_BYTES / 16; i += kThreads) reinterpret_cast<uint4*>(smem + G::OFF_Q)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < G::Q_BYTES / 16; i += kThreadsOf<BLOCK>) reinterpret_cast<uint4*>(smem + G::OFF_Q)[i] = make_uint4(0, 0, 0, 0);
   fence_proxy_async();
   if (warp == kPvWarp) {
     tmem_alloc(smem_u32(tmem_holder), G::TMEM_COLS);
@@ -456,7 +516,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   // and V stage g mod NVS, so no role needs to be told where a tile or a buffer is.
   if (warp == kProducerWarp) {
     // ============================================================== producer
-    if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); }
+    if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmK2); prefetch_tmap(&tmV2); }
     uint32_t task_it = 0, q_it = 0, k_it = 0, v_it = 0;
     bool ok = true;
     uint32_t k_armed = 0, k_parity = 0, v_armed = 0, v_parity = 0;   // per stage: parity of the last load armed on it
@@ -517,62 +577,29 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
       q_armed = true; q_armed_parity = q_it & 1;
       ++q_it;
-      // K tiles run three blocks ahead of the V tiles, like the MMAs that consume them
-      // entry q of the row's list (32 entries are fetched at a time, one per lane).  The K and the V
-      // stream of a task walk the list a few entries apart, so each has its own 32 entries:
-      // one shared set would be fetched again and again while the two sit on either side of
-      // a multiple of 32
-      int chunk_base[2] = {-64, -64}, my_idx[2] = {0, 0};
-      auto entry = [&](int q, int w) -> int {
-        if (q < chunk_base[w] || q >= chunk_base[w] + 32) {
-          chunk_base[w] = q & ~31;
-          const int e = chunk_base[w] + lane;
-          my_idx[w] = e < tk.len ? p.kv_idx[tk.lo + e] : 0;
+      int chunk_base = -64, my_idx = 0;
+      if constexpr (G::SPLIT_LOADERS) {
+        // all K tiles of the task, as fast as the ring takes them; the V tiles come from a warp of
+        // their own (64-row shapes: a tile takes twice the list entries and boxes, and one warp
+        // for both streams was the limit of the whole kernel: -27 % cycles with two)
+        for (int j = 0; j < tk.n && ok; ++j)
+          ok = load_kv_tile<G, BLOCK, true>(ctx, p, tk, p.drop_tile && t == 0 && j == 0, j, lane, sbase, BAR(B_K_FULL),
+                                            BAR(B_K_EMPTY), &tmK, &tmK2, k_it, k_armed, k_parity, chunk_base, my_idx);
+      } else {
+        // K tiles run three tiles ahead of the V tiles, like the MMAs that consume them; one warp
+        // for both streams paces the start of the next task (128-row shapes: an earlier start of
+        // the next task's loads costs more than a second loader gains, +2 % cycles)
+        int v_chunk_base = -64, v_my_idx = 0;
+        for (int j = 0; j < G::NSBUF && j < tk.n && ok; ++j)
+          ok = load_kv_tile<G, BLOCK, true>(ctx, p, tk, p.drop_tile && t == 0 && j == 0, j, lane, sbase, BAR(B_K_FULL),
+                                            BAR(B_K_EMPTY), &tmK, &tmK2, k_it, k_armed, k_parity, chunk_base, my_idx);
+        for (int j = 0; j < tk.n && ok; ++j) {
+          ok = load_kv_tile<G, BLOCK, false>(ctx, p, tk, false, j, lane, sbase, BAR(B_V_FULL), BAR(B_V_EMPTY), &tmV, &tmV2,
+                                             v_it, v_armed, v_parity, v_chunk_base, v_my_idx);
+          if (ok && j + G::NSBUF < tk.n)
+            ok = load_kv_tile<G, BLOCK, true>(ctx, p, tk, false, j + G::NSBUF, lane, sbase, BAR(B_K_FULL), BAR(B_K_EMPTY),
+                                              &tmK, &tmK2, k_it, k_armed, k_parity, chunk_base, my_idx);
         }
-        int blk = __shfl_sync(0xffffffffu, my_idx[w], q - chunk_base[w]);
-        if (blk < 0 || blk >= p.n_b) {                   // malformed list: report it and stay in range
-          if (lane == 0 && p.dev_status && atomicCAS(p.dev_status, 0, WAVEAL_ERR_BAD_MASK) == 0) {
-            p.dev_status[1] = 30; p.dev_status[2] = tk.h; p.dev_status[3] = blk;
-          }
-          blk = 0;
-        }
-        return blk;
-      };
-      auto load_tile = [&](bool is_k, int j) -> bool {
-        // the blocks of tile j: entries KB*j .. of the list (the last tile of an odd list has one)
-        const int nblk = G::KB == 1 ? 1 : min(G::KB, tk.len - G::KB * j);
-        int blk[G::KB];
-#pragma unroll
-        for (int e = 0; e < G::KB; ++e) blk[e] = e < nblk ? entry(G::KB * j + e, is_k ? 0 : 1) : 0;
-        const uint32_t it = is_k ? k_it : v_it;
-        const uint32_t nst = is_k ? (uint32_t)G::NKS : (uint32_t)G::NVS;
-        const uint32_t st = it % nst, sph = (it / nst) & 1;
-        const int b_full = (is_k ? B_K_FULL : B_V_FULL) + (int)st, b_empty = (is_k ? B_K_EMPTY : B_V_EMPTY) + (int)st;
-        if (!warp_wait(ctx, BAR(b_empty), sph ^ 1, 3)) return false;
-        // (self-test of the abort path: one tile is never requested, so its consumer's wait runs out)
-        const bool dropped = p.drop_tile && is_k && t == 0 && j == 0;
-        if (!dropped) {
-          // one lane per box: lane e*SLABS + s requests slab s of block e
-          if (lane == 0) mbar_expect_tx(BAR(b_full), (uint32_t)nblk * G::SLABS * BLOCK * 128);
-          __syncwarp();
-          const CUtensorMap* tm = is_k ? &tmK : &tmV;
-          const uint32_t dst = sbase + (is_k ? G::OFF_K : G::OFF_V) + st * G::TILE_BYTES;
-          const int e = lane / G::SLABS, sl = lane % G::SLABS;
-          int my_blk = blk[0];
-#pragma unroll
-          for (int i = 1; i < G::KB; ++i) if (e == i) my_blk = blk[i];
-          if (e < nblk)
-            tma_load_3d(dst + sl * G::KV_SLAB_BYTES + e * BLOCK * 128, tm, sl * 64, my_blk * BLOCK, tk.h, BAR(b_full));
-        }
-        if (dropped) { ++k_it; return true; }
-        if (is_k) { k_armed |= 1u << st; k_parity = (k_parity & ~(1u << st)) | (sph << st); ++k_it; }
-        else { v_armed |= 1u << st; v_parity = (v_parity & ~(1u << st)) | (sph << st); ++v_it; }
-        return true;
-      };
-      for (int j = 0; j < G::NSBUF && j < tk.n && ok; ++j) ok = load_tile(true, j);
-      for (int j = 0; j < tk.n && ok; ++j) {
-        ok = load_tile(false, j);
-        if (ok && j + G::NSBUF < tk.n) ok = load_tile(true, j + G::NSBUF);
       }
     }
     if (*abort_smem) {
@@ -591,6 +618,32 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         long long t0 = clock64();
         while (!mbar_try_wait(BAR(B_Q_FULL), q_armed_parity) && clock64() - t0 < p.wait_limit / 4) {}
       }
+    }
+  } else if (G::SPLIT_LOADERS && warp == kVLoadWarp) {
+    // ============================================================== V tile loader (64-row shapes)
+    uint32_t task_slot = 0, task_ph = 0, v_it = 0, v_armed = 0, v_parity = 0;
+    bool ok = true;
+    while (ok) {
+      ok = warp_wait(ctx, BAR(B_TASK_FULL + task_slot), task_ph, 10);
+      if (!ok) break;
+      const Task tk = tasks[task_slot];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_TASK_EMPTY + task_slot));
+      task_slot ^= 1;
+      task_ph ^= (task_slot == 0);
+      if (tk.n < 0) break;
+      int chunk_base = -64, my_idx = 0;
+      for (int j = 0; j < tk.n && ok; ++j)
+        ok = load_kv_tile<G, BLOCK, false>(ctx, p, tk, false, j, lane, sbase, BAR(B_V_FULL), BAR(B_V_EMPTY), &tmV, &tmV2,
+                                           v_it, v_armed, v_parity, chunk_base, my_idx);
+    }
+    if (*abort_smem) {
+      // leave no bulk copy in flight into this CTA's shared memory (bounded)
+      for (int st = 0; st < G::NVS; ++st)
+        if (v_armed & (1u << st)) {
+          long long t0 = clock64();
+          while (!mbar_try_wait(BAR(B_V_FULL + st), (v_parity >> st) & 1) && clock64() - t0 < p.wait_limit / 4) {}
+        }
     }
   } else if (warp == kQkWarp) {
     // ============================================================== MMA issuer 1: S = Q K^T
@@ -1129,11 +1182,13 @@ template <int BLOCK, int D>
 waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, const void* V, AttnParams& p,
                      int sms, cudaStream_t st) {
   using G = Geo<BLOCK, D>;
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq, tk, tv, tk2, tv2;
   waveal_status s;
   if ((s = make_map(&tq, Q, D, d->seq_q, d->heads, d->q_stride[0], d->q_stride[1], BLOCK, "Q")) != WAVEAL_OK) return s;
   if ((s = make_map(&tk, K, D, d->seq_kv, d->heads, d->k_stride[0], d->k_stride[1], BLOCK, "K")) != WAVEAL_OK) return s;
   if ((s = make_map(&tv, V, D, d->seq_kv, d->heads, d->v_stride[0], d->v_stride[1], BLOCK, "V")) != WAVEAL_OK) return s;
+  if ((s = make_map(&tk2, K, D, d->seq_kv, d->heads, d->k_stride[0], d->k_stride[1], 128, "K (128-row boxes)")) != WAVEAL_OK) return s;
+  if ((s = make_map(&tv2, V, D, d->seq_kv, d->heads, d->v_stride[0], d->v_stride[1], 128, "V (128-row boxes)")) != WAVEAL_OK) return s;
   WAVEAL_CUDA_OK(cudaFuncSetAttribute(k_bsattn_fwd<BLOCK, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES));
   WAVEAL_CUDA_OK(cudaFuncSetAttribute(k_bsattn_fwd<BLOCK, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES));
   WAVEAL_CUDA_OK(cudaMemsetAsync(p.ws, 0, 32, st));  // ticket counters, abort flag, redo count
@@ -1149,7 +1204,7 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   WAVEAL_CUDA_OK(cudaGetLastError());
   if (d->flags & WAVEAL_ATTN_ONLINE_MAX_ONLY) {
     p.redo_pass = 0;
-    k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
+    k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreadsOf<BLOCK>, G::SMEM_BYTES, st>>>(tq, tk, tv, tk2, tv2, p);
     WAVEAL_CUDA_OK(cudaGetLastError());
     waveal::launch_counter() = 2;
     return WAVEAL_OK;
@@ -1157,10 +1212,10 @@ waveal_status launch(const waveal_attn_desc* d, const void* Q, const void* K, co
   // first pass: reference fixed after the first two blocks of a task; second pass: the tasks the
   // first one listed (normally none: its CTAs leave at once), max of every block
   p.redo_pass = 0;
-  k_bsattn_fwd<BLOCK, D, true><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
+  k_bsattn_fwd<BLOCK, D, true><<<(unsigned)grid, kThreadsOf<BLOCK>, G::SMEM_BYTES, st>>>(tq, tk, tv, tk2, tv2, p);
   WAVEAL_CUDA_OK(cudaGetLastError());
   p.redo_pass = 1;
-  k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreads, G::SMEM_BYTES, st>>>(tq, tk, tv, p);
+  k_bsattn_fwd<BLOCK, D, false><<<(unsigned)grid, kThreadsOf<BLOCK>, G::SMEM_BYTES, st>>>(tq, tk, tv, tk2, tv2, p);
   WAVEAL_CUDA_OK(cudaGetLastError());
   waveal::launch_counter() = 3;
   return WAVEAL_OK;

@@ -337,10 +337,10 @@ def test_bounded_wait_runs_out_and_the_kernel_leaves_cleanly():
     torch.cuda.synchronize()
     dt = time.perf_counter() - t0
     code, site, cta, thread = st.tolist()
-    # whichever wait behind the lost tile ran out first: the Q K^T issuer (12), the loader's ring
-    # slot (3), the P V issuer (14) or a softmax warp (21)
-    assert code == wb.ERR_TIMEOUT and site in (3, 12, 14, 21), st.tolist()
-    assert 0 <= cta < 148 and 0 <= thread < 608
+    # whichever wait behind the lost tile ran out first: the Q K^T issuer (12), a loader's ring
+    # slot (3: K, 4: V), the P V issuer (14) or a softmax warp (21)
+    assert code == wb.ERR_TIMEOUT and site in (3, 4, 12, 14, 21), st.tolist()
+    assert 0 <= cta < 148 and 0 <= thread < 640
     assert ws.view(torch.int32)[1].item() == 1            # abort flag seen by the other thread blocks
     assert dt < 1.0, dt                                   # milliseconds, not the 2 s production limit
     # same workspace, same status words (zeroed by the caller), ordinary call
