@@ -815,6 +815,9 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const bool second = G::KB == 2 && r >= G::BQ;
       const long long q_tok = second ? (long long)tk.row2 * G::BQ + (r - G::BQ) : (long long)tk.row * G::BQ + r;
       const bool row_live = (second ? tk.row2 >= 0 : r < G::BQ) && q_tok < p.seq_q;
+      // rows 64..127 of a tile that no second block shares hold nothing: their warps only keep
+      // the barriers of the tile going (each output row of an MMA depends on its own row of S / P alone)
+      const bool idle = G::KB == 2 && quad >= 2 && tk.row2 < 0;
       __nv_bfloat16* o_ptr = p.O + (size_t)tk.h * p.o_stride_h + (size_t)q_tok * p.o_stride_t + part * G::CO;
       if (tk.n == 0) {
         if (row_live) {
@@ -831,6 +834,12 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if ((int)par == team) {
           ok = warp_wait(ctx, BAR(B_S_FULL + sb), (s_phase >> sb) & 1u, 21);
           if (!ok) break;
+          if (idle) {
+            if (lane == 0) mbar_arrive(BAR(B_P_FULL + sb * 2 + half));
+            s_phase ^= 1u << sb;
+            if (++sb == (uint32_t)G::NSBUF) sb = 0;
+            continue;
+          }
           tc_fence_after();
           const uint32_t s_addr = tmem_base + lane_addr + sb * G::S_STRIDE + half * G::HC;
           const bool ragged = j == tk.n - 1 && tk.tail_valid < G::BK;
@@ -975,7 +984,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
         // both teams count every block
         s_phase ^= 1u << sb;
-        if (!(FAST && j >= 2)) mx_phase ^= 1u << par;   // one flip per arrival on that parity's barrier
+        if (!(FAST && j >= 2) && !idle) mx_phase ^= 1u << par;   // one flip per arrival on that parity's barrier
         if (++sb == (uint32_t)G::NSBUF) sb = 0;
       }
       if (!ok) break;
