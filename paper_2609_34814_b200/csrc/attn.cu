@@ -8,9 +8,12 @@
 // SM, take tickets from a global counter, so a freed SM starts the next row of the list at
 // once - the streaming "wave" behaviour of Section 2.3 that the schedule is built for.
 //
-// Structure of one CTA (608 threads):
+// Structure of one CTA (608 threads; 640 in the kernels of the 64-row blocks):
 //   warp 0      producer: takes tickets, publishes tasks, issues TMA loads of the Q tile and
 //               of the K and V tiles (128-byte-swizzled slabs) into two shared-memory rings
+//   warp 19     64-row blocks only: requests the V tiles instead of warp 0 (a tile of that shape
+//               takes two list entries and up to four boxes; one warp for both streams was the
+//               limit of the whole kernel there)
 //   warp 18     MMA issuer 1: S_j = Q K_j^T (operands in shared memory) into one of three S
 //               buffers in tensor memory, up to three blocks ahead of the softmax
 //   warp 1      MMA issuer 2: O += P_j V_j (P read from tensor memory, where it lies over the
