@@ -251,6 +251,7 @@ def run_waveal(args, cfg):
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_ev)
     step_cycles = int(aws_words[4].item())          # SM cycles of the attention launch of the last timed step
     step_pairs = int(aws_words[6].item())           # query-block pairs that shared a tile in it (64-row blocks)
+    step_tiles = int(aws_words[7].item())           # 128-row x 128-key MMA tiles it ran
     check_status()
     flops_all = wd.sum_over_ranks(flops, dev) if world > 1 else flops
     value = flops_all / (ms_per_step * 1e-3) / 1e12
@@ -411,6 +412,7 @@ def run_waveal(args, cfg):
                      "frac_of_sustained": achieved / pk["bf16_sustained"] if pk["bf16_sustained"] else None,
                      "frac_of_datasheet_2250": achieved / 2250.0,
                      "kernel_ms": attn_ms, "kernel_sm_cycles": step_cycles, "tiles_shared_by_two_blocks": step_pairs,
+                     "mma_tiles": step_tiles, "mma_tile_fill": (pairs * B * B / (step_tiles * 128.0 * 128.0)) if step_tiles else None,
                      "traffic": traffic,
                      "traffic_source": "ncu, one launch of this workload (profiles/)" if traffic else None},
         "counters": {"source": "profiles/k_bsattn_fwd_%s.txt (ncu, one launch per order)" % cfg.name, **ctr} if ctr else None,

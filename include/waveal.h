@@ -205,7 +205,8 @@ typedef struct waveal_attn_desc {
 /* Bytes of device workspace waveal_bsattn_fwd needs: 32 bytes of counters (int32 words: ticket
  * counter, abort flag, number of tasks computed twice, ticket counter of the second launch,
  * length of the first and of the second launch in SM cycles = the largest lifetime of a thread
- * block, number of query-block pairs that shared a tile, one spare), 8 bytes per (head, query block) for the list of tasks to compute again and
+ * block, number of query-block pairs that shared a tile, number of 128-row x 128-key tiles the call runs),
+ * 8 bytes per (head, query block) for the list of tasks to compute again and
  * 32 bytes per (head, query block) for the table that maps a ticket to its task.  The counters
  * are live state of the call (tickets are drawn from them): calls that may overlap on the GPU
  * must not share a workspace.  Host-only. */

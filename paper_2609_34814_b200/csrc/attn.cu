@@ -1132,6 +1132,7 @@ __global__ void k_task_table(AttnParams p, int block_k, Task* table) {
       }
     }
   }
+  if (tk.n > 0) atomicAdd(&p.ws[7], tk.n);    // word 7: KV tiles (128 rows x 128 keys) this call runs
   table[t] = tk;
 }
 
