@@ -993,6 +993,12 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       if (!ok) break;
       // ---- epilogue: O / l at the original row position; l = the four partial sums of the row
       // brought to the final reference (the larger of the two teams', references never shrink)
+      // (the partial sums are final once the thread's last tile is done: publish them before the
+      // wait for the last P V, so that nothing but the load of O stands between that MMA and the
+      // first one of the next task)
+      exb[part * 128 + r] = make_float2(m_ref, l_run);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_EX + quad));
       ok = warp_wait(ctx, BAR(B_O_FULL), o_it & 1, 23);
       if (!ok) break;
       ++o_it;
@@ -1006,11 +1012,15 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (G::KB == 2 && tk.row2 >= 0) { p.ws[10 + 2 * e] = tk.h; p.ws[11 + 2 * e] = tk.row2; }   // computed again one by one
         redo_flag[rslot] = 0;
       }
-      exb[part * 128 + r] = make_float2(m_ref, l_run);
+      uint32_t ov[G::CO];
+      static_assert(G::CO == 32 || G::CO == 16, "a quarter of head_dim 128 or 64");
+      if constexpr (G::CO == 32) { WAVEAL_TMEM_LD32(o_row + part * G::CO, ov, 0); WAVEAL_TMEM_WAIT_LD32(ov, 0); }
+      else { WAVEAL_TMEM_LD16(o_row + part * G::CO, ov, 0); WAVEAL_TMEM_WAIT_LD16(ov, 0); }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_O_FREE));
       // the other three warps of this lane quadrant have written their parts: a bounded wait
       // like every other, so that a warp whose partners gave up does not stay behind
-      __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_EX + quad));
       ok = warp_wait(ctx, BAR(B_EX + quad), (o_it & 1) ^ 1, 25);
       if (!ok) break;
       const float2 e00 = exb[0 * 128 + r], e01 = exb[1 * 128 + r], e10 = exb[2 * 128 + r], e11 = exb[3 * 128 + r];
@@ -1020,13 +1030,6 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const float a1 = (m1 == -INFINITY) ? 0.f : ex2(m1 - m_all);
       const float l_tot = a0 * (e00.y + e01.y) + a1 * (e10.y + e11.y);
       const float inv_l = 1.0019531f / l_tot;    // the sums carry the centring factor 1 + 2^-9
-      uint32_t ov[G::CO];
-      static_assert(G::CO == 32 || G::CO == 16, "a quarter of head_dim 128 or 64");
-      if constexpr (G::CO == 32) { WAVEAL_TMEM_LD32(o_row + part * G::CO, ov, 0); WAVEAL_TMEM_WAIT_LD32(ov, 0); }
-      else { WAVEAL_TMEM_LD16(o_row + part * G::CO, ov, 0); WAVEAL_TMEM_WAIT_LD16(ov, 0); }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_O_FREE));
       if (row_live) {
 #pragma unroll
         for (int c = 0; c < G::CO; c += 8) {
