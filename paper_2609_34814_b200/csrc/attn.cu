@@ -246,6 +246,13 @@ __device__ __forceinline__ void ex2_fma2(float& e0, float& e1, float s0, float s
         "r"(taddr)                                                                               \
       : "memory")
 
+// one 32-byte store (the address must be 32-byte aligned)
+__device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t* w) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(ptr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
+}
+
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -524,34 +531,51 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     bool ok = true;
     uint32_t k_armed = 0, k_parity = 0, v_armed = 0, v_parity = 0;   // per stage: parity of the last load armed on it
     bool q_armed = false; uint32_t q_armed_parity = 0;
+    // the next task: a ticket from the global counter and the task it stands for (n = -1: none left)
+    auto draw = [&](long long& t_out) -> Task {
+      for (;;) {
+        long long t = 0, n_tasks = p.total_tasks;
+        if (lane == 0) {
+          if (p.redo_pass) n_tasks = min((long long)p.ws[2], p.total_tasks);   // written by the first pass
+          // (volatile: another SM raises the flag while this kernel runs; a cached copy would hide it)
+          t = (*reinterpret_cast<volatile int*>(&p.ws[1]) != 0) ? n_tasks
+                                                               : (long long)(unsigned)atomicAdd(&p.ws[p.redo_pass ? 3 : 0], 1);
+        }
+        t = __shfl_sync(0xffffffffu, t, 0);
+        n_tasks = __shfl_sync(0xffffffffu, n_tasks, 0);
+        t_out = t;
+        Task tk{};
+        if (t >= n_tasks) {
+          tk.n = -1;
+        } else if (!p.redo_pass) {
+          // one 32-byte load behind the ticket instead of a chain through three lists
+          const uint4* e = reinterpret_cast<const uint4*>(p.table + t);
+          const uint4 a = e[0], b = e[1];
+          tk.h = (int)a.x; tk.row = (int)a.y; tk.lo = (int)a.z; tk.n = (int)a.w; tk.tail_valid = (int)b.x; tk.len = (int)b.y;
+          tk.row2 = (int)b.z;
+          if (tk.n == kAbsorbed) continue;          // second block of a pair: computed with its partner
+        } else {
+          int h = p.ws[8 + 2 * t], row = p.ws[9 + 2 * t];
+          if (h < 0 || h >= p.heads) h = 0;
+          if (row < 0 || row >= p.m_b) row = 0;
+          int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
+          tk.h = h; tk.row = row; tk.lo = lo; tk.row2 = -1;
+          fill_tiles(tk, max(hi - lo, 0), BLOCK, hi > lo ? p.kv_idx[hi - 1] : 0, p.n_b, p.seq_kv);
+        }
+        return tk;
+      }
+    };
+    // The ticket of the next task is drawn a few tiles before the current task's last loads are
+    // requested, while this warp would wait for a ring stage anyway: the round trips of the
+    // counter and of the table entry (~2,000 cycles) then no longer stand between the end of a
+    // task and the request for the next Q tile.
+    constexpr int kDrawAhead = 3;
+    long long t = 0, t_next = 0;
+    Task tk_next = draw(t_next);
     while (ok) {
-      long long t = 0, n_tasks = p.total_tasks;
-      if (lane == 0) {
-        if (p.redo_pass) n_tasks = min((long long)p.ws[2], p.total_tasks);   // written by the first pass
-        // (volatile: another SM raises the flag while this kernel runs; a cached copy would hide it)
-        t = (*reinterpret_cast<volatile int*>(&p.ws[1]) != 0) ? n_tasks
-                                                             : (long long)(unsigned)atomicAdd(&p.ws[p.redo_pass ? 3 : 0], 1);
-      }
-      t = __shfl_sync(0xffffffffu, t, 0);
-      n_tasks = __shfl_sync(0xffffffffu, n_tasks, 0);
-      Task tk{};
-      if (t >= n_tasks) {
-        tk.n = -1;
-      } else if (!p.redo_pass) {
-        // one 32-byte load behind the ticket instead of a chain through three lists
-        const uint4* e = reinterpret_cast<const uint4*>(p.table + t);
-        const uint4 a = e[0], b = e[1];
-        tk.h = (int)a.x; tk.row = (int)a.y; tk.lo = (int)a.z; tk.n = (int)a.w; tk.tail_valid = (int)b.x; tk.len = (int)b.y;
-        tk.row2 = (int)b.z;
-        if (tk.n == kAbsorbed) continue;          // second block of a pair: computed with its partner
-      } else {
-        int h = p.ws[8 + 2 * t], row = p.ws[9 + 2 * t];
-        if (h < 0 || h >= p.heads) h = 0;
-        if (row < 0 || row >= p.m_b) row = 0;
-        int lo = p.row_ptr[(size_t)h * p.m_b + row], hi = p.row_ptr[(size_t)h * p.m_b + row + 1];
-        tk.h = h; tk.row = row; tk.lo = lo; tk.row2 = -1;
-        fill_tiles(tk, max(hi - lo, 0), BLOCK, hi > lo ? p.kv_idx[hi - 1] : 0, p.n_b, p.seq_kv);
-      }
+      Task tk = tk_next;
+      t = t_next;
+      bool drawn = false;
       const uint32_t slot = task_it & 1, ph = (task_it >> 1) & 1;
       ok = warp_wait(ctx, BAR(B_TASK_EMPTY + slot), ph ^ 1, 1);
       if (!ok) break;
@@ -561,6 +585,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
       ++task_it;
       if (tk.n < 0) break;
+      if (tk.n <= kDrawAhead) { tk_next = draw(t_next); drawn = true; }
       if (tk.n == 0) continue;
       // Q tile
       ok = warp_wait(ctx, BAR(B_Q_EMPTY), (q_it & 1) ^ 1, 2);
@@ -585,9 +610,11 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         // all K tiles of the task, as fast as the ring takes them; the V tiles come from a warp of
         // their own (64-row shapes: a tile takes twice the list entries and boxes, and one warp
         // for both streams was the limit of the whole kernel: -27 % cycles with two)
-        for (int j = 0; j < tk.n && ok; ++j)
+        for (int j = 0; j < tk.n && ok; ++j) {
+          if (!drawn && j >= tk.n - kDrawAhead) { tk_next = draw(t_next); drawn = true; }
           ok = load_kv_tile<G, BLOCK, true>(ctx, p, tk, p.drop_tile && t == 0 && j == 0, j, lane, sbase, BAR(B_K_FULL),
                                             BAR(B_K_EMPTY), &tmK, &tmK2, k_it, k_armed, k_parity, chunk_base, my_idx);
+        }
       } else {
         // K tiles run three tiles ahead of the V tiles, like the MMAs that consume them; one warp
         // for both streams paces the start of the next task (128-row shapes: an earlier start of
@@ -597,6 +624,7 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           ok = load_kv_tile<G, BLOCK, true>(ctx, p, tk, p.drop_tile && t == 0 && j == 0, j, lane, sbase, BAR(B_K_FULL),
                                             BAR(B_K_EMPTY), &tmK, &tmK2, k_it, k_armed, k_parity, chunk_base, my_idx);
         for (int j = 0; j < tk.n && ok; ++j) {
+          if (!drawn && j >= tk.n - kDrawAhead) { tk_next = draw(t_next); drawn = true; }
           ok = load_kv_tile<G, BLOCK, false>(ctx, p, tk, false, j, lane, sbase, BAR(B_V_FULL), BAR(B_V_EMPTY), &tmV, &tmV2,
                                              v_it, v_armed, v_parity, v_chunk_base, v_my_idx);
           if (ok && j + G::NSBUF < tk.n)
@@ -1031,16 +1059,22 @@ k_bsattn_fwd(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       const float l_tot = a0 * (e00.y + e01.y) + a1 * (e10.y + e11.y);
       const float inv_l = 1.0019531f / l_tot;    // the sums carry the centring factor 1 + 2^-9
       if (row_live) {
+        // a thread holds a piece of one row, so a store instruction of a warp touches 32 rows:
+        // its cost in the memory pipe is per row, not per byte.  32-byte stores halve the number
+        // of instructions where the row piece is 32-byte aligned (else 16-byte stores)
+        uint32_t w[G::CO / 2];
 #pragma unroll
-        for (int c = 0; c < G::CO; c += 8) {
-          uint32_t w[4];
+        for (int c = 0; c < G::CO; c += 2) {
+          __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(ov[c]) * inv_l, __uint_as_float(ov[c + 1]) * inv_l);
+          w[c / 2] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        if ((reinterpret_cast<uintptr_t>(o_ptr) & 31) == 0) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(ov[c + 2 * e]) * inv_l,
-                                                      __uint_as_float(ov[c + 2 * e + 1]) * inv_l);
-            w[e] = *reinterpret_cast<uint32_t*>(&b2);
-          }
-          *reinterpret_cast<uint4*>(o_ptr + c) = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int c = 0; c < G::CO / 2; c += 8) st_global_v8(o_ptr + 2 * c, w + c);
+        } else {
+#pragma unroll
+          for (int c = 0; c < G::CO / 2; c += 4)
+            *reinterpret_cast<uint4*>(o_ptr + 2 * c) = make_uint4(w[c], w[c + 1], w[c + 2], w[c + 3]);
         }
         if (p.lse && part == 0) p.lse[(size_t)tk.h * p.seq_q + q_tok] = (m_all + log2f(l_tot) - 0.0028150156f) * 0.6931471805599453f;
       }

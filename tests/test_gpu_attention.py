@@ -109,6 +109,23 @@ def test_empty_rows_scale_and_strides():
         assert np.abs(lse[li].cpu().numpy()[fin] - ref_lse[fin]).max() < 2e-3
 
 
+def test_output_rows_at_16_byte_alignment_only():
+    """O whose rows start at 16-byte but not 32-byte boundaries (the least the interface asks for):
+    the kernel's narrower stores must write the same bits as the 32-byte ones."""
+    cfg = _small("wan480p", 2, 2)
+    w = Workload(cfg)
+    base, st = run_attention(w)
+    assert st[0] == 0
+    n = 2 * cfg.seq_pad * cfg.head_dim
+    buf = torch.full((n + 8,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    o = buf[8:].view(2, cfg.seq_pad, cfg.head_dim)
+    assert o.data_ptr() % 32 == 16
+    o, st = run_attention(w, out=o)
+    assert st[0] == 0
+    assert torch.equal(o[:, :cfg.seq], base[:, :cfg.seq])
+    assert torch.isnan(buf[:8]).all()
+
+
 def test_closed_forms_on_gpu():
     cfg = _small("wan480p", 2, 1)
     w = Workload(cfg)
